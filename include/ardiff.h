@@ -1,0 +1,162 @@
+/*
+ * ardiff.h -- C ABI of the entropy-gated few-step diffusion-head hot path (B200, sm_100a).
+ *
+ * Two calls make the path:
+ *   ardiff_entropy_gate  per-token entropy of the softmax-normalised shallow-feature row,
+ *                        threshold, stream-compacted ascending list of surviving token ids;
+ *   ardiff_head_sample   K Euler flow steps of the AdaLN residual-MLP head, conditioned on
+ *                        each surviving token's AR hidden state, from caller-supplied noise.
+ *
+ * Conventions for every call
+ *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are
+ *     ordinary host memory. The caller owns every buffer it passes.
+ *   - bf16 data is passed as raw 16-bit patterns (uint16_t / void*).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). All
+ *     device work is enqueued on it; calls return without waiting unless stated otherwise.
+ *   - return value: 0 on success, a negative ARDIFF_ERR_* otherwise. Nothing throws,
+ *     aborts or traps the device. Invalid arguments are rejected before any launch.
+ */
+#ifndef ARDIFF_H
+#define ARDIFF_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ARDIFF_OK 0
+#define ARDIFF_ERR_NULL (-1)        /* a required pointer is NULL                           */
+#define ARDIFF_ERR_SHAPE (-2)       /* a size is negative, zero where it may not be, or too big */
+#define ARDIFF_ERR_ALIGN (-3)       /* a pointer or row pitch misses its alignment rule      */
+#define ARDIFF_ERR_UNSUPPORTED (-4) /* a shape the kernels do not cover (see each call)      */
+#define ARDIFF_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed                     */
+#define ARDIFF_ERR_TIMEOUT (-6)     /* a bounded device-side wait ran out (results invalid)  */
+#define ARDIFF_ERR_NOMEM (-7)       /* an allocation inside a create call failed             */
+
+const char* ardiff_strerror(int code);
+/* major*10000 + minor*100 + patch */
+int ardiff_version(void);
+
+/* ---------------------------------------------------------------------------------------
+ * Entropy gate + stream compaction.
+ *
+ * Operation (the paper's entropy indicator: "Entropy-Informed Speculative Decoding",
+ * equation for L_entropy, and the supplementary "Entropy Calculation Logic"; the test is
+ * Algorithm 1's "if H^s < tau_ent"): for every token i, Omega = softmax(feat[i, :]) over
+ * the d channels, H_i = -sum_c Omega_c ln Omega_c (natural log, zero-probability terms
+ * contribute 0), keep_i = (H_i >= tau). A row that holds NaN, +inf or only -inf gives
+ * H_i = NaN and is dropped.
+ *
+ *   feat   dev  bf16 [n][d] row-major (pre-softmax values), 16-byte aligned when d % 8 == 0
+ *   n      tokens, 0 <= n < 2^31;  d channels per token, 1 <= d <= 65536
+ *   tau    threshold (compared in fp32)
+ *   mask   dev  uint8 [n]  out: 1 = keep, 0 = dropped
+ *   idx    dev  int32 [n]  out: the first *count entries are the kept token ids, ascending
+ *   count  dev  int32 [1]  out: number of kept tokens (stays on the device)
+ *   entropy (the _ex form) dev float [n] out, or NULL: H_i as computed
+ *
+ * Rows are read once from HBM (d <= 8192 and d % 8 == 0: registers hold the row; other d
+ * take a slower two-pass kernel). Uses a small per-device scratch (per-block counts) that
+ * the library allocates on the first call on each device: make that first call outside
+ * any stream capture. n == 0 is valid (writes *count = 0).
+ * ------------------------------------------------------------------------------------- */
+int ardiff_entropy_gate(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask,
+                        int32_t* idx, int32_t* count, void* stream);
+
+int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask,
+                           int32_t* idx, int32_t* count, float* entropy, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Diffusion / flow head.
+ *
+ * Operation (the head call "x = Diff_theta(x_t | t, z)" of the AR+Diffusion hybrid
+ * paradigm, sampled in "extremely few steps" from noise fixed up front as in Algorithm 1's
+ * "Initialize"): for every survivor j < *count, with i = idx[j], z = cond[i], x = noise[i]:
+ *   c = Wc z + bc
+ *   for k in 0..K-1:
+ *     s = SiLU(c + temb(t_k)),   temb(t) = Wt2 SiLU(Wt1 e(t) + bt1) + bt2,
+ *         e(t) = [cos(1000 t w_f) | sin(1000 t w_f)], w_f = 10000^(-f/(F/2)), f < F/2
+ *     h = Win x + bin
+ *     for b in 0..L-1:  (shift, scale, gate) = Wmod[b] s + bmod[b]
+ *                       u = LN(h) * (1 + scale) + shift          LN: eps 1e-6, no affine
+ *                       h = h + gate * (W2[b] SiLU(W1[b] u + b1[b]) + b2[b])
+ *     (shift, scale) = Wfm s + bfm ;  v = Wout (LN(h) * (1 + scale) + shift) + bout
+ *     x = x + (t_{k+1} - t_k) v
+ *   out[i] = x
+ * Matrix products take bf16 operands with fp32 accumulation on the tensor cores; the
+ * residual stream h, the state x, LayerNorm statistics and SiLU are fp32.
+ * ------------------------------------------------------------------------------------- */
+typedef struct ardiff_head ardiff_head; /* opaque; owns device copies of the weights + scratch */
+
+typedef struct {
+    int32_t C;      /* token (latent) dim: multiple of 16, 16 <= C <= 64                   */
+    int32_t Dc;     /* conditioning dim: multiple of 64                                    */
+    int32_t W;      /* head width: multiple of 256, <= 4096                                */
+    int32_t L;      /* residual blocks, 1 <= L <= 64                                       */
+    int32_t F;      /* time-embedding size (even), <= 1024                                 */
+    int32_t K_max;  /* largest K a later ardiff_head_sample may ask for, <= 64             */
+    int64_t max_tokens; /* largest *count a later ardiff_head_sample may meet              */
+} ardiff_head_desc;
+
+/* HOST pointers, bf16 bit patterns, Linear layout [out][in] row-major, biases [out]. */
+typedef struct {
+    const uint16_t *Wc, *bc;     /* [W][Dc], [W]                                          */
+    const uint16_t *Wt1, *bt1;   /* [W][F],  [W]                                          */
+    const uint16_t *Wt2, *bt2;   /* [W][W],  [W]                                          */
+    const uint16_t *Win, *bin;   /* [W][C],  [W]                                          */
+    const uint16_t *Wmod, *bmod; /* [L][3W][W], [L][3W]   rows: shift | scale | gate      */
+    const uint16_t *W1, *b1;     /* [L][W][W], [L][W]                                     */
+    const uint16_t *W2, *b2;     /* [L][W][W], [L][W]                                     */
+    const uint16_t *Wfm, *bfm;   /* [2W][W], [2W]         rows: shift | scale             */
+    const uint16_t *Wout, *bout; /* [C][W],  [C]                                          */
+} ardiff_head_host_weights;
+
+/*
+ * Packs the weights into the kernels' tile layout on the current device and allocates
+ * the head's scratch (a fixed-size activation workspace sized to stay L2-resident plus
+ * max_tokens/128 progress counters). Synchronous; the only head call that allocates.
+ * Errors: ERR_NULL, ERR_SHAPE / ERR_UNSUPPORTED for dims outside the ranges above,
+ * ERR_NOMEM, ERR_CUDA (also when the device is not compute capability 10.x).
+ */
+int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_head_host_weights* weights,
+                       ardiff_head** head_out);
+
+/* Frees everything create allocated. Waits for the device first. NULL is accepted. */
+int ardiff_head_destroy(ardiff_head* head);
+
+/*
+ *   head     from ardiff_head_create (same device)
+ *   cond     dev  bf16 [n][Dc] row-major, 16-byte aligned
+ *   noise    dev  float [n][C]
+ *   t_sched  HOST float [K+1]: t_0 .. t_K (read before the call returns)
+ *   K        steps, 0 <= K <= K_max (K == 0 copies noise rows to out rows)
+ *   idx      dev  int32: token ids of the survivors (as written by the gate; any order,
+ *                 each a valid row of cond / noise / out, no duplicates)
+ *   count    dev  int32 [1]: number of survivors; read on the device, never on the host;
+ *                 values above max_tokens are clamped to max_tokens (and flagged in the
+ *                 status word as ARDIFF_ERR_SHAPE)
+ *   out      dev  float [n][C]: rows idx[j] are written, all other rows are left untouched
+ * One persistent cooperative kernel walks a static schedule of GEMM tiles; tiles wait for
+ * their producers on device-side counters with bounded spins. If a wait runs out the
+ * kernel finishes early, the results are invalid and ardiff_head_status reports
+ * ARDIFF_ERR_TIMEOUT. Calls on one head must not overlap on the device (they share its
+ * scratch): enqueue them on one stream or order them with events.
+ */
+int ardiff_head_sample(const ardiff_head* head, const void* cond, const float* noise,
+                       const float* t_sched, int32_t K, const int32_t* idx, const int32_t* count,
+                       float* out, void* stream);
+
+/* Waits for `stream`, then returns the head's device status word: ARDIFF_OK, or
+ * ARDIFF_ERR_TIMEOUT if any bounded wait of an earlier sample call ran out, or
+ * ARDIFF_ERR_SHAPE if *count exceeded max_tokens. Clears it. */
+int ardiff_head_status(ardiff_head* head, void* stream);
+
+/* Number of kernel launches the last ardiff_head_sample / ardiff_entropy_gate call on this
+ * thread enqueued (for launch accounting by benchmarks). */
+int ardiff_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARDIFF_H */

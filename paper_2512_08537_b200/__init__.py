@@ -1,0 +1,171 @@
+"""Python binding of libardiff (the C ABI declared in include/ardiff.h).
+
+Argument marshalling only: every step of the hot path runs in the CUDA kernels of the shared
+library. torch is used for device memory and streams. There is no CPU fallback: if the library
+cannot be loaded, or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libardiff.so")
+_lib = None
+
+ARDIFF_OK = 0
+ARDIFF_ERR_NULL, ARDIFF_ERR_SHAPE, ARDIFF_ERR_ALIGN, ARDIFF_ERR_UNSUPPORTED = -1, -2, -3, -4
+ARDIFF_ERR_CUDA, ARDIFF_ERR_TIMEOUT, ARDIFF_ERR_NOMEM = -5, -6, -7
+
+_WEIGHT_FIELDS = ["Wc", "bc", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wmod", "bmod",
+                  "W1", "b1", "W2", "b2", "Wfm", "bfm", "Wout", "bout"]
+
+
+class ArdiffError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class HeadDesc(ctypes.Structure):
+    _fields_ = [("C", ctypes.c_int32), ("Dc", ctypes.c_int32), ("W", ctypes.c_int32),
+                ("L", ctypes.c_int32), ("F", ctypes.c_int32), ("K_max", ctypes.c_int32),
+                ("max_tokens", ctypes.c_int64)]
+
+
+class HeadHostWeights(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_void_p) for k in _WEIGHT_FIELDS]
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libardiff.so (building it with nvcc first if it is missing). Raises if it cannot."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            from . import build as _build
+            _build.build()
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float
+        L.ardiff_strerror.restype = ctypes.c_char_p
+        L.ardiff_strerror.argtypes = [ctypes.c_int]
+        L.ardiff_version.restype = ctypes.c_int
+        L.ardiff_last_launch_count.restype = ctypes.c_int
+        L.ardiff_entropy_gate.restype = ctypes.c_int
+        L.ardiff_entropy_gate.argtypes = [vp, i64, i32, f32, vp, vp, vp, vp]
+        L.ardiff_entropy_gate_ex.restype = ctypes.c_int
+        L.ardiff_entropy_gate_ex.argtypes = [vp, i64, i32, f32, vp, vp, vp, vp, vp]
+        if hasattr(L, "ardiff_head_create"):
+            L.ardiff_head_create.restype = ctypes.c_int
+            L.ardiff_head_create.argtypes = [ctypes.POINTER(HeadDesc), ctypes.POINTER(HeadHostWeights),
+                                             ctypes.POINTER(vp)]
+            L.ardiff_head_destroy.restype = ctypes.c_int
+            L.ardiff_head_destroy.argtypes = [vp]
+            L.ardiff_head_sample.restype = ctypes.c_int
+            L.ardiff_head_sample.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
+            L.ardiff_head_status.restype = ctypes.c_int
+            L.ardiff_head_status.argtypes = [vp, vp]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().ardiff_strerror(int(code)).decode()
+
+
+def version() -> int:
+    return int(lib().ardiff_version())
+
+
+def last_launch_count() -> int:
+    return int(lib().ardiff_last_launch_count())
+
+
+def _check(rc: int, where: str):
+    if rc != ARDIFF_OK:
+        raise ArdiffError(rc, where)
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def ardiff_entropy_gate(feat, tau: float, mask=None, idx=None, count=None, entropy=None,
+                        want_entropy: bool = False, stream=None):
+    """Entropy gate + compaction on `feat` (torch bf16 CUDA tensor [n, d]).
+
+    Returns (mask u8 [n], idx i32 [n], count i32 [1], entropy f32 [n] or None); outputs are
+    allocated here unless passed in. Nothing is synchronised.
+    """
+    import torch
+    assert feat.is_cuda and feat.dtype == torch.bfloat16 and feat.dim() == 2 and feat.is_contiguous()
+    n, d = feat.shape
+    dev = feat.device
+    if mask is None:
+        mask = torch.empty((n,), dtype=torch.uint8, device=dev)
+    if idx is None:
+        idx = torch.empty((max(n, 1),), dtype=torch.int32, device=dev)
+    if count is None:
+        count = torch.empty((1,), dtype=torch.int32, device=dev)
+    if entropy is None and want_entropy:
+        entropy = torch.empty((n,), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ardiff_entropy_gate_ex(
+            feat.data_ptr(), n, d, float(tau), mask.data_ptr(), idx.data_ptr(), count.data_ptr(),
+            entropy.data_ptr() if entropy is not None else None, _stream_ptr(stream))
+    _check(rc, "ardiff_entropy_gate")
+    return mask, idx, count, entropy
+
+
+class Head:
+    """Owns an ardiff_head handle (device weights + scratch)."""
+
+    def __init__(self, C: int, Dc: int, W: int, L: int, F: int, K_max: int, max_tokens: int,
+                 weights: Dict[str, "object"]):
+        import numpy as np
+        L_ = lib()
+        if not hasattr(L_, "ardiff_head_create"):
+            raise RuntimeError("libardiff.so was built without the head")
+        self.desc = HeadDesc(C=C, Dc=Dc, W=W, L=L, F=F, K_max=K_max, max_tokens=max_tokens)
+        keep = {k: np.ascontiguousarray(weights[k]) for k in _WEIGHT_FIELDS}
+        for k, a in keep.items():
+            assert a.dtype == np.uint16, f"{k}: bf16 bit patterns (uint16) expected"
+        hw = HeadHostWeights(**{k: keep[k].ctypes.data for k in _WEIGHT_FIELDS})
+        h = ctypes.c_void_p()
+        _check(L_.ardiff_head_create(ctypes.byref(self.desc), ctypes.byref(hw), ctypes.byref(h)),
+               "ardiff_head_create")
+        self._h = h
+
+    def ardiff_head_sample(self, cond, noise, t_sched, idx, count, out, stream=None):
+        """K = len(t_sched)-1 steps for the survivors idx[0..*count); writes rows of `out`."""
+        import numpy as np
+        import torch
+        assert cond.is_cuda and cond.dtype == torch.bfloat16 and cond.is_contiguous()
+        assert noise.is_cuda and noise.dtype == torch.float32 and noise.is_contiguous()
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+        assert idx.dtype == torch.int32 and count.dtype == torch.int32
+        ts = np.ascontiguousarray(t_sched, dtype=np.float32)
+        K = ts.shape[0] - 1
+        with torch.cuda.device(cond.device):
+            rc = lib().ardiff_head_sample(self._h, cond.data_ptr(), noise.data_ptr(), ts.ctypes.data, K,
+                                          idx.data_ptr(), count.data_ptr(), out.data_ptr(),
+                                          _stream_ptr(stream))
+        _check(rc, "ardiff_head_sample")
+        return out
+
+    def status(self, stream=None) -> int:
+        return int(lib().ardiff_head_status(self._h, _stream_ptr(stream)))
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().ardiff_head_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,165 @@
+"""GPU parity of the entropy gate + compaction against the fp64 oracle, through the C ABI.
+
+Agreement bar: entropy within 1e-3 absolute; mask equal for every token whose oracle entropy is
+at least 1e-4 away from tau; idx/count bit-exact against the GPU's own mask (ascending positions)
+and, when no token lies in the band, bit-exact against the oracle's.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+import paper_2512_08537_b200 as ardiff
+from gpu_util import dev_bf16, require_cuda
+
+pytestmark = pytest.mark.gpu
+
+ENT_TOL = 1e-3
+BAND = 1e-4
+
+
+def run_gate(bits, tau):
+    feat = dev_bf16(bits)
+    mask, idx, count, ent = ardiff.ardiff_entropy_gate(feat, tau, want_entropy=True)
+    torch.cuda.synchronize()
+    c = int(count.item())
+    return mask.cpu().numpy(), idx.cpu().numpy()[:c], c, ent.cpu().numpy()
+
+
+def check(bits, tau):
+    H, mask_o, idx_o, count_o = oracle.gate(bits, tau)
+    mask_g, idx_g, count_g, ent_g = run_gate(bits, tau)
+    nan_o = np.isnan(H)
+    assert np.array_equal(np.isnan(ent_g), nan_o)
+    assert np.all(np.abs(ent_g[~nan_o] - H[~nan_o]) <= ENT_TOL)
+    off_band = nan_o | (np.abs(H - float(np.float32(tau))) >= BAND)
+    assert np.array_equal(mask_g[off_band], mask_o[off_band])
+    assert count_g == int(mask_g.sum())
+    assert np.array_equal(idx_g, np.flatnonzero(mask_g).astype(np.int32))
+    if off_band.all():
+        assert count_g == count_o and np.array_equal(idx_g, idx_o)
+    return H, mask_g, count_g
+
+
+def quantile_tau(H, q):
+    """Midpoint between neighbouring order statistics, so the band around tau is usually empty."""
+    Hs = np.sort(H[~np.isnan(H)])
+    k = int(round(q * len(Hs)))
+    if k <= 0:
+        return -1.0
+    if k >= len(Hs):
+        return float(Hs[-1]) + 1.0
+    return 0.5 * (float(Hs[k - 1]) + float(Hs[k]))
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4"])
+def test_workload_configs(name):
+    wl = synth.workload(name)
+    bits = synth.features(wl)
+    H = oracle.entropy(bits)
+    tau = quantile_tau(H, wl.filter_q)
+    _, mask_g, count_g = check(bits, tau)
+    assert abs(count_g - round((1 - wl.filter_q) * wl.n)) <= 16
+
+
+@pytest.mark.parametrize("n", [1, 7, 8, 31, 33, 129, 1000, 4099])
+@pytest.mark.parametrize("d", [8, 16, 256, 264, 768, 1024, 2048, 3072, 5120, 6144, 8192])
+def test_shapes_vector_path(n, d):
+    if n * d > 4099 * 1024 and n > 129:
+        n = 129
+    wl = synth.workload("cfg2", n=n, d=d, seed=1000 + d)
+    bits = synth.features(wl)
+    H = oracle.entropy(bits)
+    for q in (0.0, 0.5, 1.0):
+        check(bits, quantile_tau(H, q))
+
+
+@pytest.mark.parametrize("d", [1, 2, 7, 12, 777, 1001, 8200, 16384])
+def test_shapes_generic_path(d):
+    wl = synth.workload("cfg2", n=67, d=d, seed=2000 + d)
+    bits = synth.features(wl)
+    H = oracle.entropy(bits)
+    for q in (0.0, 0.4):
+        check(bits, quantile_tau(H, q))
+
+
+def test_empty_input_writes_zero_count():
+    dev = require_cuda()
+    feat = torch.empty((0, 64), dtype=torch.bfloat16, device=dev)
+    count = torch.full((1,), 77, dtype=torch.int32, device=dev)
+    ardiff.ardiff_entropy_gate(feat, 0.5, count=count)
+    torch.cuda.synchronize()
+    assert int(count.item()) == 0
+
+
+def test_special_rows_minus_inf_nan_inf_uniform_onehot():
+    d = 512
+    x = np.zeros((8, d), np.float32)
+    x[1, 5] = 100.0                       # one-hot limit -> 0
+    x[2, :100] = -np.inf                  # -inf channels contribute nothing: H = ln(412)
+    x[3, :] = -np.inf                     # undefined -> dropped
+    x[4, 17] = np.nan                     # dropped
+    x[5, 300] = np.inf                    # dropped
+    x[6, :] = 3.0                         # uniform: ln d
+    x[7, ::2] = 1.5                       # two-level closed form
+    bits = synth.f32_to_bf16(x)
+    H, mask_g, count_g = check(bits, 0.5)
+    assert abs(H[0] - np.log(d)) < 1e-12 and abs(H[2] - np.log(412)) < 1e-12
+    assert list(mask_g) == [1, 0, 1, 0, 0, 0, 1, 1]
+    # same rows through the generic kernel (d not a multiple of 8)
+    check(synth.f32_to_bf16(x[:, :509]), 0.5)
+
+
+def test_tau_extremes_keep_all_and_drop_all():
+    wl = synth.workload("cfg2", n=3000)
+    bits = synth.features(wl)
+    _, m_all, c_all = check(bits, -1.0)
+    assert c_all == 3000
+    _, m_none, c_none = check(bits, 100.0)
+    assert c_none == 0
+
+
+def test_bad_arguments_are_rejected_without_launching():
+    dev = require_cuda()
+    lib = ardiff.lib()
+    buf = torch.zeros(4096, dtype=torch.uint8, device=dev)
+    p = buf.data_ptr()
+    assert lib.ardiff_entropy_gate(None, 4, 8, 0.0, p, p, p, None) == ardiff.ARDIFF_ERR_NULL
+    assert lib.ardiff_entropy_gate(p, 4, 8, 0.0, p, p, None, None) == ardiff.ARDIFF_ERR_NULL
+    assert lib.ardiff_entropy_gate(p, -1, 8, 0.0, p, p, p, None) == ardiff.ARDIFF_ERR_SHAPE
+    assert lib.ardiff_entropy_gate(p, 4, 0, 0.0, p, p, p, None) == ardiff.ARDIFF_ERR_SHAPE
+    assert lib.ardiff_entropy_gate(p + 2, 4, 8, 0.0, p, p, p, None) == ardiff.ARDIFF_ERR_ALIGN
+    torch.cuda.synchronize()
+
+
+def test_full_size_gate_stress_sampled_rows_and_properties():
+    """2^20 x 5120 (10.7 GB): features are generated and uploaded in slabs; the oracle checks a
+    sample of rows one by one, the rest is checked through properties that hold at any size."""
+    dev = require_cuda()
+    wl = synth.workload("cfg5")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 14 * 2**30:
+        pytest.fail("needs 14 GB of free device memory")
+    feat = torch.empty((wl.n, wl.d), dtype=torch.bfloat16, device=dev)
+    slab = 32768
+    for r0 in range(0, wl.n, slab):
+        feat[r0:r0 + slab] = dev_bf16(synth.features(wl, r0, slab))
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([np.arange(0, 64), np.arange(wl.n - 64, wl.n),
+                                     rng.integers(0, wl.n, size=4096)]))
+    H_s = np.array([oracle.entropy(synth.features(wl, int(r), 1))[0] for r in rows])
+    for q in (0.0, 0.1, 0.5, 0.9, 0.99):
+        tau = quantile_tau(H_s, q)
+        mask, idx, count, ent = ardiff.ardiff_entropy_gate(feat, tau, want_entropy=True)
+        torch.cuda.synchronize()
+        c = int(count.item())
+        ent_s = ent[torch.from_numpy(rows).to(dev)].cpu().numpy()
+        mask_s = mask[torch.from_numpy(rows).to(dev)].cpu().numpy()
+        assert np.all(np.abs(ent_s - H_s) <= ENT_TOL)
+        off = np.abs(H_s - float(np.float32(tau))) >= BAND
+        assert np.array_equal(mask_s[off], (H_s >= float(np.float32(tau))).astype(np.uint8)[off])
+        assert c == int(mask.sum().item())
+        want_idx = torch.nonzero(mask, as_tuple=False).flatten().to(torch.int32)
+        assert torch.equal(idx[:c], want_idx)
+        assert abs(c / wl.n - (1 - q)) < 0.03
