@@ -1,0 +1,1112 @@
+// K-step AdaLN residual-MLP flow head for sm_100a: one persistent cooperative kernel.
+//
+// What it computes (per surviving token; see include/ardiff.h for the formulas): the head call
+// x = Diff_theta(x_t | t, z) of the AR+Diffusion hybrid, conditioned on the token's AR hidden
+// state z and on t, sampled with K Euler flow steps from caller-supplied noise.
+//
+// How: every matrix product of the head is cut into tiles of 128 tokens x 256 output columns.
+// Each tile is one "item": TMA streams the bf16 A (activations) and B (weights) K-slices into a
+// 4-stage shared-memory ring, one thread issues tcgen05.mma (bf16 x bf16 -> fp32) into one of
+// two 256-column TMEM accumulators, and four epilogue warps read the accumulator back with
+// tcgen05.ld and apply the fused tail of that layer (bias, SiLU, LayerNorm+modulation, gated
+// residual, LayerNorm statistics, Euler update, scatter) while the next item's MMAs already run.
+// All items of all layers and steps form one static list ordered so that the activations of a
+// group of token tiles stay in L2; CTA c takes items c, c+grid, ... . A tile of layer l needs all
+// column tiles of layer l-1 of the same 128 tokens: that is tracked with one progress counter per
+// token tile (release/acquire at gpu scope, bounded spins).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "../../include/ardiff.h"
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int BM = 128;           // tokens per tile
+constexpr int BN = 256;           // output columns per tile (UMMA N)
+constexpr int BK = 64;            // K slice per pipeline stage (128 bytes of bf16: one swizzle row)
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+constexpr int NUM_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int EPI_THREADS = 128;
+constexpr int XB_COLS = 64;       // x is fed to the in-projection as bf16, K padded to one slice
+constexpr int KMAX = 64;
+constexpr uint64_t kWaitLimitNs = 4000000000ull;   // a bounded wait gives up after 4 s
+constexpr uint64_t kDrainLimitNs = 200000000ull;   // waits for own copies in flight at exit
+
+enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_MOD, OP_G1, OP_G2, OP_FMOD, OP_OUT };
+enum MapId : int { MAP_Z = 0, MAP_XB, MAP_S, MAP_U, MAP_A, MAP_WC, MAP_WIN, MAP_WCAT, MAP_WOUT, MAP_COUNT };
+
+struct StepOp {
+    int type;      // OpType
+    int ntiles;    // column tiles of this op per token tile
+    int cum;       // column tiles of the ops before it within one step
+    int map_a, map_b;
+    int b_row0;    // first row of this op's weights in the B matrix
+    int kblocks;   // K / 64
+    int umma_n;    // 256, or C for the out-projection
+    int block;     // residual block index (or -1)
+};
+
+struct HeadParams {
+    int C, Dc, W, L, K, NT, TG, slots;      // NT = W/256, slots = 2*TG token tiles of scratch
+    int T_pro, T_step, T_chain, n_step_ops;
+    int max_tokens;
+    const StepOp* step_ops;
+    const CUtensorMap* maps;
+    const bf16* cond;
+    const float* noise;
+    const int* idx;
+    const int* count;
+    float* out;
+    bf16 *z, *xb, *s, *u, *a, *g;
+    float *x, *c, *h;
+    float2* stats;
+    const float *bias_cat, *bc, *bin, *temb;
+    int* counters;
+    int* status;
+    int* abort_flag;
+    float dt[KMAX];
+};
+
+struct Item {
+    int type, abs_m, slot_row0, nt, k, prior;
+    int map_a, map_b, b_row, kblocks, umma_n, block;
+};
+
+// ------------------------------------------------------------------------------------------
+// device helpers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void raise_timeout(const HeadParams& P) {
+    atomicExch(P.abort_flag, 1);
+    atomicCAS(P.status, 0, ARDIFF_ERR_TIMEOUT);
+}
+
+// bounded wait on an mbarrier phase; false = gave up (abort raised or seen)
+__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const HeadParams& P,
+                                          uint64_t limit_ns = kWaitLimitNs) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    uint64_t t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((it & 127u) == 0) {
+            if (ptx::ld_relaxed_gpu(P.abort_flag) != 0) return false;
+            const uint64_t now = ptx::globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) {
+                raise_timeout(P);
+                return false;
+            }
+        }
+    }
+}
+
+// bounded wait until *ctr >= need (acquire); one thread calls it
+__device__ __forceinline__ bool wait_counter(const int* ctr, int need, const HeadParams& P) {
+    if (ptx::ld_acquire_gpu(ctr) >= need) return true;
+    uint64_t t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (ptx::ld_acquire_gpu(ctr) >= need) return true;
+        if (it > 8) __nanosleep(64);
+        if ((it & 63u) == 0) {
+            if (ptx::ld_relaxed_gpu(P.abort_flag) != 0) return false;
+            const uint64_t now = ptx::globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) {
+                raise_timeout(P);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ bool epi_any(bool pred) {  // OR over the 128 epilogue threads
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 2, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return r != 0;
+}
+
+__device__ __forceinline__ float silu_f(float a) { return __fdividef(a, 1.0f + __expf(-a)); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ void decode_item(const HeadParams& P, int MT, long long item, Item& it) {
+    const long long per_group = (long long)P.TG * P.T_chain;
+    const int grp = (int)(item / per_group);
+    int r = (int)(item - (long long)grp * per_group);
+    const int m0 = grp * P.TG;
+    const int mtg = min(P.TG, MT - m0);
+    const int pro = mtg * P.T_pro;
+    int m;
+    if (r < pro) {
+        it.k = 0;
+        it.block = -1;
+        if (r < mtg) {
+            it.type = OP_GATHER; m = r; it.nt = 0; it.prior = 0;
+            it.map_a = it.map_b = 0; it.b_row = 0; it.kblocks = 0; it.umma_n = 0;
+        } else {
+            r -= mtg;
+            m = r / P.NT;
+            it.nt = r - m * P.NT;
+            it.type = OP_COND; it.prior = 1;
+            it.map_a = MAP_Z; it.map_b = MAP_WC; it.b_row = it.nt * BN;
+            it.kblocks = P.Dc / BK; it.umma_n = BN;
+        }
+    } else {
+        r -= pro;
+        const int per_step = mtg * P.T_step;
+        it.k = r / per_step;
+        r -= it.k * per_step;
+        int o = 0;
+        while (o + 1 < P.n_step_ops && __ldg(&P.step_ops[o + 1].cum) * mtg <= r) ++o;
+        const StepOp op = P.step_ops[o];
+        const int q = r - op.cum * mtg;
+        m = q / op.ntiles;
+        it.nt = q - m * op.ntiles;
+        it.type = op.type;
+        it.prior = P.T_pro + it.k * P.T_step + op.cum;
+        it.map_a = op.map_a; it.map_b = op.map_b;
+        it.b_row = op.b_row0 + it.nt * BN;
+        it.kblocks = op.kblocks; it.umma_n = op.umma_n; it.block = op.block;
+    }
+    it.abs_m = m0 + m;
+    it.slot_row0 = (it.abs_m % P.slots) * BM;
+}
+
+// ------------------------------------------------------------------------------------------
+// epilogues. Thread `row` (0..127) of the tile owns TMEM lane `row`; `tacc` addresses its lane
+// at column 0 of the accumulator. Each handles 32 columns per tcgen05.ld.
+// ------------------------------------------------------------------------------------------
+struct Stats {
+    float p, sd, sq;
+    __device__ __forceinline__ void init(float first) { p = first; sd = 0.f; sq = 0.f; }
+    __device__ __forceinline__ void add(float v) { const float e = v - p; sd += e; sq = fmaf(e, e, sq); }
+    __device__ __forceinline__ float2 finish(int n) const {
+        const float inv = 1.0f / (float)n;
+        const float mean = p + sd * inv;
+        const float m2 = fmaxf(sq - sd * sd * inv, 0.f);
+        return make_float2(mean, m2);
+    }
+};
+
+__device__ __forceinline__ void load_acc32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    ptx::tmem_ld_32x32b_x32(taddr, r);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void add_bias32(float (&v)[32], const float* __restrict__ bias) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        const float4 b = __ldg(reinterpret_cast<const float4*>(bias + i));
+        v[i] += b.x; v[i + 1] += b.y; v[i + 2] += b.z; v[i + 3] += b.w;
+    }
+}
+
+__device__ __forceinline__ void store_bf16_32(bf16* dst, const float (&v)[32]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        uint4 w;
+        w.x = pack_bf16x2(v[i], v[i + 1]);
+        w.y = pack_bf16x2(v[i + 2], v[i + 3]);
+        w.z = pack_bf16x2(v[i + 4], v[i + 5]);
+        w.w = pack_bf16x2(v[i + 6], v[i + 7]);
+        ptx::st_u4(dst + i, w);
+    }
+}
+
+__device__ __forceinline__ void store_f32_32(float* dst, const float (&v)[32]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) ptx::st_f4(dst + i, make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+}
+
+__device__ __forceinline__ void load_f32_32(const float* src, float (&v)[32]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        const float4 t = ptx::ldcg_f4(src + i);
+        v[i] = t.x; v[i + 1] = t.y; v[i + 2] = t.z; v[i + 3] = t.w;
+    }
+}
+
+__device__ __forceinline__ void load_bf16_32(const bf16* src, float (&v)[32]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        const uint4 w = ptx::ldcg_u4(src + i);
+        v[i] = bf16lo(w.x); v[i + 1] = bf16hi(w.x); v[i + 2] = bf16lo(w.y); v[i + 3] = bf16hi(w.y);
+        v[i + 4] = bf16lo(w.z); v[i + 5] = bf16hi(w.z); v[i + 6] = bf16lo(w.w); v[i + 7] = bf16hi(w.w);
+    }
+}
+
+// c = acc + bc
+__device__ __forceinline__ void epi_cond(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
+    const int col0 = it.nt * BN;
+    float* crow = P.c + (size_t)grow * P.W + col0;
+#pragma unroll 1
+    for (int cc = 0; cc < BN / 32; ++cc) {
+        float v[32];
+        load_acc32(tacc + cc * 32, v);
+        add_bias32(v, P.bc + col0 + cc * 32);
+        store_f32_32(crow + cc * 32, v);
+    }
+}
+
+// h = acc + bin ; LN partial statistics ; s = SiLU(c + temb_k)
+__device__ __forceinline__ void epi_in(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
+    const int col0 = it.nt * BN;
+    float* hrow = P.h + (size_t)grow * P.W + col0;
+    const float* crow = P.c + (size_t)grow * P.W + col0;
+    bf16* srow = P.s + (size_t)grow * P.W + col0;
+    const float* temb = P.temb + (size_t)it.k * P.W + col0;
+    Stats st;
+#pragma unroll 1
+    for (int cc = 0; cc < BN / 32; ++cc) {
+        float v[32];
+        load_acc32(tacc + cc * 32, v);
+        add_bias32(v, P.bin + col0 + cc * 32);
+        if (cc == 0) st.init(v[0]);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) st.add(v[i]);
+        store_f32_32(hrow + cc * 32, v);
+        float cv[32];
+        load_f32_32(crow + cc * 32, cv);
+        add_bias32(cv, temb + cc * 32);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) cv[i] = silu_f(cv[i]);
+        store_bf16_32(srow + cc * 32, cv);
+    }
+    P.stats[(size_t)grow * P.NT + it.nt] = st.finish(BN);
+}
+
+__device__ __forceinline__ void row_mean_rstd(const HeadParams& P, int grow, float& mean, float& rstd) {
+    const float2* sp = P.stats + (size_t)grow * P.NT;
+    float msum = 0.f;
+    for (int t = 0; t < P.NT; ++t) msum += ptx::ldcg_f2(sp + t).x;
+    mean = msum / (float)P.NT;
+    float m2 = 0.f;
+    for (int t = 0; t < P.NT; ++t) {
+        const float2 v = ptx::ldcg_f2(sp + t);
+        const float dm = v.x - mean;
+        m2 += v.y + (float)BN * dm * dm;
+    }
+    rstd = rsqrtf(m2 / (float)P.W + 1e-6f);
+}
+
+// shift/scale tile: accumulator columns [0,128) = shift, [128,256) = scale of h columns
+// [nt*128, nt*128+128):  u = LN(h) * (1 + scale) + shift
+__device__ __forceinline__ void epi_mod_ss(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
+    float mean, rstd;
+    row_mean_rstd(P, grow, mean, rstd);
+    const int hcol0 = it.nt * 128;
+    const float* hrow = P.h + (size_t)grow * P.W + hcol0;
+    bf16* urow = P.u + (size_t)grow * P.W + hcol0;
+    const float* bias = P.bias_cat + it.b_row;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+        float sh[32], sc[32], hv[32];
+        load_acc32(tacc + cc * 32, sh);
+        load_acc32(tacc + 128 + cc * 32, sc);
+        add_bias32(sh, bias + cc * 32);
+        add_bias32(sc, bias + 128 + cc * 32);
+        load_f32_32(hrow + cc * 32, hv);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], sh[i]);
+        store_bf16_32(urow + cc * 32, hv);
+    }
+}
+
+// gate tile: g = acc + bias (columns [ (nt - W/128)*256, +256 ) of the block's gate)
+__device__ __forceinline__ void epi_mod_g(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
+    const int col0 = (it.nt - P.W / 128) * BN;
+    bf16* grow_p = P.g + (size_t)grow * P.W + col0;
+    const float* bias = P.bias_cat + it.b_row;
+#pragma unroll 1
+    for (int cc = 0; cc < BN / 32; ++cc) {
+        float v[32];
+        load_acc32(tacc + cc * 32, v);
+        add_bias32(v, bias + cc * 32);
+        store_bf16_32(grow_p + cc * 32, v);
+    }
+}
+
+// a = SiLU(acc + b1)
+__device__ __forceinline__ void epi_g1(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
+    const int col0 = it.nt * BN;
+    bf16* arow = P.a + (size_t)grow * P.W + col0;
+    const float* bias = P.bias_cat + it.b_row;
+#pragma unroll 1
+    for (int cc = 0; cc < BN / 32; ++cc) {
+        float v[32];
+        load_acc32(tacc + cc * 32, v);
+        add_bias32(v, bias + cc * 32);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = silu_f(v[i]);
+        store_bf16_32(arow + cc * 32, v);
+    }
+}
+
+// h += g * (acc + b2) ; LN partial statistics of the new h
+__device__ __forceinline__ void epi_g2(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
+    const int col0 = it.nt * BN;
+    float* hrow = P.h + (size_t)grow * P.W + col0;
+    const bf16* grow_p = P.g + (size_t)grow * P.W + col0;
+    const float* bias = P.bias_cat + it.b_row;
+    Stats st;
+#pragma unroll 1
+    for (int cc = 0; cc < BN / 32; ++cc) {
+        float v[32], gv[32], hv[32];
+        load_acc32(tacc + cc * 32, v);
+        add_bias32(v, bias + cc * 32);
+        load_bf16_32(grow_p + cc * 32, gv);
+        load_f32_32(hrow + cc * 32, hv);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) hv[i] = fmaf(gv[i], v[i], hv[i]);
+        if (cc == 0) st.init(hv[0]);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) st.add(hv[i]);
+        store_f32_32(hrow + cc * 32, hv);
+    }
+    P.stats[(size_t)grow * P.NT + it.nt] = st.finish(BN);
+}
+
+// v = acc + bout ; x += dt_k v ; bf16 copy for the next in-projection ; last step: out[idx[j]] = x
+__device__ __forceinline__ void epi_out(const HeadParams& P, const Item& it, uint32_t tacc, int grow,
+                                        int j, int count) {
+    const float dt = P.dt[it.k];
+    float* xrow = P.x + (size_t)grow * P.C;
+    bf16* xbrow = P.xb + (size_t)grow * XB_COLS;
+    const float* bias = P.bias_cat + it.b_row;
+    const bool last = (it.k == P.K - 1);
+    float* orow = nullptr;
+    if (last && j < count) orow = P.out + (size_t)__ldg(P.idx + j) * P.C;
+    for (int cc = 0; cc < P.C / 16; ++cc) {
+        uint32_t r[16];
+        ptx::tmem_ld_32x32b_x16(tacc + cc * 16, r);
+        ptx::tmem_ld_wait();
+        float xn[16];
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + cc * 16 + i));
+            const float4 xo = ptx::ldcg_f4(xrow + cc * 16 + i);
+            xn[i] = fmaf(dt, __uint_as_float(r[i]) + b.x, xo.x);
+            xn[i + 1] = fmaf(dt, __uint_as_float(r[i + 1]) + b.y, xo.y);
+            xn[i + 2] = fmaf(dt, __uint_as_float(r[i + 2]) + b.z, xo.z);
+            xn[i + 3] = fmaf(dt, __uint_as_float(r[i + 3]) + b.w, xo.w);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+            const float4 v4 = make_float4(xn[i], xn[i + 1], xn[i + 2], xn[i + 3]);
+            ptx::st_f4(xrow + cc * 16 + i, v4);
+            if (orow) ptx::st_f4(orow + cc * 16 + i, v4);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; i += 8) {
+            uint4 w;
+            w.x = pack_bf16x2(xn[i], xn[i + 1]);
+            w.y = pack_bf16x2(xn[i + 2], xn[i + 3]);
+            w.z = pack_bf16x2(xn[i + 4], xn[i + 5]);
+            w.w = pack_bf16x2(xn[i + 6], xn[i + 7]);
+            ptx::st_u4(xbrow + cc * 16 + i, w);
+        }
+    }
+}
+
+// rows of this token tile: z = cond[idx[j]], x = noise[idx[j]], xb = bf16(x); rows past count: 0
+__device__ __forceinline__ void gather_rows(const HeadParams& P, const Item& it, int ewarp, int lane,
+                                            int count) {
+    const int chunks = P.Dc / 8;  // 16-byte chunks per cond row
+    for (int r = ewarp * 32; r < ewarp * 32 + 32; ++r) {
+        const int j = it.abs_m * BM + r;
+        const int grow = it.slot_row0 + r;
+        const bool valid = j < count;
+        const size_t tok = valid ? (size_t)__ldg(P.idx + j) : 0;
+        const uint4* src = reinterpret_cast<const uint4*>(P.cond + tok * P.Dc);
+        uint4* dst = reinterpret_cast<uint4*>(P.z + (size_t)grow * P.Dc);
+        for (int c = lane; c < chunks; c += 32) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (valid) v = __ldg(src + c);
+            dst[c] = v;
+        }
+        for (int c = lane; c < P.C; c += 32) {
+            const float xv = valid ? __ldg(P.noise + tok * P.C + c) : 0.f;
+            P.x[(size_t)grow * P.C + c] = xv;
+            P.xb[(size_t)grow * XB_COLS + c] = __float2bfloat16_rn(xv);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// the persistent kernel
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_constant__ HeadParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = ptx::smem_u32(smem);
+    const uint32_t bars = smem_base + STAGES * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 5));
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    int count = __ldg(P.count);
+    if (count > P.max_tokens) {
+        count = P.max_tokens;
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(P.status, 0, ARDIFF_ERR_SHAPE);
+    }
+    if (count < 0) count = 0;
+    const int MT = (count + BM - 1) / BM;
+    const long long total = (long long)MT * P.T_chain;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull_bar(b), 1);
+            ptx::mbar_init(tempty_bar(b), 4);
+        }
+        ptx::mbar_init(drain_bar, 1);
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t issued = 0, issued_parity = 0;
+        for (long long item = blockIdx.x; item < total; item += gridDim.x) {
+            Item it;
+            decode_item(P, MT, item, it);
+            if (it.type == OP_GATHER) continue;
+            bool ok = true;
+            if (lane == 0) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            ptx::fence_proxy_async();
+            const void* map_a = P.maps + it.map_a;
+            const void* map_b = P.maps + it.map_b;
+            const uint32_t tx = A_BYTES + (uint32_t)it.umma_n * BK * 2;
+            for (int kb = 0; kb < it.kblocks; ++kb) {
+                ok = wait_mbar(empty_bar(stage), phase ^ 1u, P);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                    ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                    ptx::tma_load_2d(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
+                    ptx::tma_load_2d(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row);
+                }
+                issued |= 1u << stage;
+                issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+        }
+        // own copies in flight: every stage's last issue must have landed before the CTA exits
+        for (int s = 0; s < STAGES; ++s)
+            if (issued & (1u << s)) wait_mbar(full_bar(s), (issued_parity >> s) & 1u, P, kDrainLimitNs);
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t acc_iter = 0;
+        for (long long item = blockIdx.x; item < total; item += gridDim.x) {
+            Item it;
+            decode_item(P, MT, item, it);
+            if (it.type == OP_GATHER) continue;
+            const uint32_t buf = acc_iter & 1u;
+            const uint32_t acc_phase = (acc_iter >> 1) & 1u;
+            bool ok = wait_mbar(tempty_bar(buf), acc_phase ^ 1u, P);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * BN;
+            const uint32_t idesc = ptx::idesc_bf16_f32(BM, (uint32_t)it.umma_n);
+            for (int kb = 0; kb < it.kblocks; ++kb) {
+                ok = wait_mbar(full_bar(stage), phase, P);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ptx::tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                    const uint64_t da = ptx::smem_desc_sw128(sa);
+                    const uint64_t db = ptx::smem_desc_sw128(sa + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        ptx::mma_f16_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
+                    ptx::mma_commit(empty_bar(stage));
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (lane == 0) ptx::mma_commit(tfull_bar(buf));
+            __syncwarp();
+            ++acc_iter;
+        }
+        // all MMAs this thread issued must be done before TMEM is freed
+        if (lane == 0) ptx::mma_commit(drain_bar);
+        __syncwarp();
+        wait_mbar(drain_bar, 0, P, kDrainLimitNs);
+    } else {
+        // ---------------- epilogue warps ----------------
+        const int ewarp = warp - 2;           // 0..3
+        const int quarter = warp & 3;         // TMEM lane quarter this warp may read
+        const int row = quarter * 32 + lane;  // row of the tile owned by this thread
+        const bool leader = (threadIdx.x == 64);
+        uint32_t acc_iter = 0;
+        for (long long item = blockIdx.x; item < total; item += gridDim.x) {
+            Item it;
+            decode_item(P, MT, item, it);
+            if (it.type == OP_GATHER) {
+                bool ok = true;
+                if (leader && it.abs_m >= P.slots)
+                    ok = wait_counter(P.counters + (it.abs_m - P.slots), P.T_chain, P);
+                if (epi_any(!ok)) break;
+                gather_rows(P, it, ewarp, lane, count);
+            } else {
+                const uint32_t buf = acc_iter & 1u;
+                const uint32_t acc_phase = (acc_iter >> 1) & 1u;
+                bool ok = wait_mbar(tfull_bar(buf), acc_phase, P);
+                // the operands of this item arrived, so its producers are done; take the acquire
+                // in this thread too before reading what other CTAs wrote
+                if (ok && leader) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
+                if (epi_any(!ok)) break;
+                ptx::tc_fence_after();
+                const uint32_t tacc = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
+                const int grow = it.slot_row0 + row;
+                switch (it.type) {
+                    case OP_COND: epi_cond(P, it, tacc, grow); break;
+                    case OP_IN: epi_in(P, it, tacc, grow); break;
+                    case OP_MOD:
+                        if (it.nt < P.W / 128) epi_mod_ss(P, it, tacc, grow);
+                        else epi_mod_g(P, it, tacc, grow);
+                        break;
+                    case OP_FMOD: epi_mod_ss(P, it, tacc, grow); break;
+                    case OP_G1: epi_g1(P, it, tacc, grow); break;
+                    case OP_G2: epi_g2(P, it, tacc, grow); break;
+                    default: epi_out(P, it, tacc, grow, it.abs_m * BM + row, count); break;
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
+                ++acc_iter;
+            }
+            // publish: this item's global writes, then one tick of the token tile's counter
+            __threadfence();
+            ptx::fence_proxy_async();
+            ptx::named_barrier_sync(1, EPI_THREADS);
+            if (leader) ptx::red_release_gpu_add(P.counters + it.abs_m, 1);
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// small kernels: time embedding MLP, K = 0 copy
+// ------------------------------------------------------------------------------------------
+struct TimeArgs {
+    float t[KMAX];
+};
+
+// hidden[k][o] = SiLU(Wt1[o] . e(t_k) + bt1[o]); one warp per output
+__global__ void __launch_bounds__(256) temb_hidden_kernel(const bf16* __restrict__ Wt1,
+                                                         const float* __restrict__ bt1, int W, int F,
+                                                         TimeArgs ta, float* __restrict__ hidden) {
+    extern __shared__ float e_s[];
+    const int k = blockIdx.y;
+    const int half = F / 2;
+    for (int f = threadIdx.x; f < half; f += blockDim.x) {
+        const double w = exp(-log(10000.0) * (double)f / (double)half);
+        const double arg = 1000.0 * (double)ta.t[k] * w;
+        double sn, cs;
+        sincos(arg, &sn, &cs);
+        e_s[f] = (float)cs;
+        e_s[half + f] = (float)sn;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int o = blockIdx.x * 8 + warp;
+    if (o >= W) return;
+    const bf16* wr = Wt1 + (size_t)o * F;
+    float acc = 0.f;
+    for (int i = lane; i < F; i += 32) acc = fmaf(__bfloat162float(wr[i]), e_s[i], acc);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+    if (lane == 0) {
+        const float a = acc + bt1[o];
+        hidden[(size_t)k * W + o] = a / (1.0f + expf(-a));
+    }
+}
+
+// temb[k][o] = Wt2[o] . hidden[k] + bt2[o]
+__global__ void __launch_bounds__(256) temb_out_kernel(const bf16* __restrict__ Wt2,
+                                                      const float* __restrict__ bt2, int W,
+                                                      const float* __restrict__ hidden,
+                                                      float* __restrict__ temb) {
+    const int k = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int o = blockIdx.x * 8 + warp;
+    if (o >= W) return;
+    const bf16* wr = Wt2 + (size_t)o * W;
+    const float* hk = hidden + (size_t)k * W;
+    float acc = 0.f;
+    for (int i = lane * 2; i < W; i += 64) {
+        const __nv_bfloat162 w2 = *reinterpret_cast<const __nv_bfloat162*>(wr + i);
+        acc = fmaf(__low2float(w2), hk[i], acc);
+        acc = fmaf(__high2float(w2), hk[i + 1], acc);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+    if (lane == 0) temb[(size_t)k * W + o] = acc + bt2[o];
+}
+
+__global__ void copy_noise_rows_kernel(const float* __restrict__ noise, const int* __restrict__ idx,
+                                       const int* __restrict__ count, int max_tokens, int C,
+                                       float* __restrict__ out) {
+    int cnt = min(*count, max_tokens);
+    const long long total = (long long)cnt * C;
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const int j = (int)(e / C), c = (int)(e % C);
+        const size_t tok = (size_t)idx[j];
+        out[tok * C + c] = noise[tok * C + c];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major [rows][cols] tensor, box = [box_rows][64 cols], 128-byte swizzle
+bool make_map(CUtensorMap* m, void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline float bf16_bits_to_float(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+}  // namespace
+
+struct ardiff_head {
+    ardiff_head_desc d;
+    int device, n_sm, grid;
+    int NT, TG, slots, T_pro, T_step, T_chain, n_step_ops;
+    int64_t max_tiles;
+    std::vector<void*> allocs;
+    // device
+    bf16 *Wcat, *Wc, *Win, *Wt1, *Wt2;
+    float *bias_cat, *bc, *bin, *bt1, *bt2, *temb, *temb_hidden;
+    bf16 *z, *xb, *s, *u, *a, *g;
+    float *x, *c, *h;
+    float2* stats;
+    int *counters, *status;  // status[0] = status word, status[1] = abort flag
+    StepOp* step_ops;
+    CUtensorMap* maps;
+};
+
+namespace {
+
+template <typename T>
+int dev_alloc(ardiff_head* H, T** p, size_t count, bool zero) {
+    void* q = nullptr;
+    if (cudaMalloc(&q, count * sizeof(T) + 256) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ARDIFF_ERR_NOMEM;
+    }
+    H->allocs.push_back(q);
+    if (zero && cudaMemset(q, 0, count * sizeof(T) + 256) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    *p = reinterpret_cast<T*>(q);
+    return ARDIFF_OK;
+}
+
+int upload(void* dst, const void* src, size_t bytes) {
+    return cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice) == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+}
+
+int upload_bias(float* dst, const uint16_t* src, size_t n) {
+    std::vector<float> tmp(n);
+    for (size_t i = 0; i < n; ++i) tmp[i] = bf16_bits_to_float(src[i]);
+    return upload(dst, tmp.data(), n * sizeof(float));
+}
+
+void free_all(ardiff_head* H) {
+    for (void* p : H->allocs) cudaFree(p);
+    H->allocs.clear();
+}
+
+int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    if (!v || !*v) return dflt;
+    return atoi(v);
+}
+
+}  // namespace
+
+#define TRY(expr)                   \
+    do {                            \
+        int _rc = (expr);           \
+        if (_rc != ARDIFF_OK) {     \
+            free_all(H);            \
+            delete H;               \
+            return _rc;             \
+        }                           \
+    } while (0)
+
+extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_head_host_weights* w,
+                                  ardiff_head** head_out) {
+    if (!desc || !w || !head_out) return ARDIFF_ERR_NULL;
+    *head_out = nullptr;
+    const ardiff_head_desc d = *desc;
+    if (d.C < 16 || d.C > 64 || d.Dc < 64 || d.W < 256 || d.W > 4096 || d.L < 1 || d.L > 64 || d.F < 2 ||
+        d.F > 1024 || d.K_max < 0 || d.K_max > KMAX || d.max_tokens < 0 || d.max_tokens >= ((int64_t)1 << 31) - 256)
+        return ARDIFF_ERR_SHAPE;
+    if (d.C % 16 || d.Dc % 64 || d.W % 256 || d.F % 2) return ARDIFF_ERR_UNSUPPORTED;
+    const void* ptrs[] = {w->Wc, w->bc, w->Wt1, w->bt1, w->Wt2, w->bt2, w->Win, w->bin, w->Wmod, w->bmod,
+                          w->W1, w->b1, w->W2, w->b2, w->Wfm, w->bfm, w->Wout, w->bout};
+    for (const void* p : ptrs)
+        if (!p) return ARDIFF_ERR_NULL;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess)
+        return ARDIFF_ERR_CUDA;
+    if (prop.major != 10) return ARDIFF_ERR_CUDA;
+    if (!get_encode_fn()) return ARDIFF_ERR_CUDA;
+
+    ardiff_head* H = new ardiff_head();
+    H->d = d;
+    H->device = dev;
+    H->n_sm = prop.multiProcessorCount;
+    const int W = d.W, C = d.C, Dc = d.Dc, L = d.L;
+    H->NT = W / BN;
+    H->T_pro = 1 + H->NT;
+    H->T_step = H->NT * (3 + 5 * L) + 1;
+    H->n_step_ops = 3 * L + 3;
+    H->max_tiles = (d.max_tokens + BM - 1) / BM;
+    if (H->max_tiles < 1) H->max_tiles = 1;
+
+    // grid: one CTA per SM, all co-resident (cooperative launch)
+    if (cudaFuncSetAttribute(head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+        delete H;
+        return ARDIFF_ERR_CUDA;
+    }
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, head_kernel, NUM_THREADS, SMEM_BYTES) != cudaSuccess ||
+        per_sm < 1) {
+        delete H;
+        return ARDIFF_ERR_CUDA;
+    }
+    H->grid = env_int("ARDIFF_HEAD_GRID", H->n_sm);
+    if (H->grid < 1 || H->grid > H->n_sm) H->grid = H->n_sm;
+
+    // token tiles per group: enough column tiles per layer to keep every CTA busy while the
+    // layer before it drains (about 1.5 grids of items), capped by what exists
+    int tg = (3 * H->grid / 2 + H->NT - 1) / H->NT;
+    tg = env_int("ARDIFF_HEAD_TG", tg);
+    if (tg < 1) tg = 1;
+    if ((int64_t)tg > H->max_tiles) tg = (int)H->max_tiles;
+    H->TG = tg;
+    H->slots = 2 * tg;
+    const size_t R = (size_t)H->slots * BM;
+
+    // ---- pack the weights: one K-major matrix [rows][W] for every W-input layer ----
+    const size_t blk_rows = (size_t)5 * W;
+    const size_t fm_row0 = blk_rows * L, out_row0 = fm_row0 + 2 * (size_t)W;
+    const size_t cat_rows = out_row0 + C;
+    {
+        std::vector<uint16_t> cat(cat_rows * W);
+        std::vector<float> bias(cat_rows);
+        auto put = [&](size_t dst_row, const uint16_t* Wsrc, const uint16_t* bsrc, size_t src_row, size_t nrows) {
+            memcpy(&cat[dst_row * W], Wsrc + src_row * W, nrows * W * 2);
+            for (size_t i = 0; i < nrows; ++i) bias[dst_row + i] = bf16_bits_to_float(bsrc[src_row + i]);
+        };
+        auto put_shift_scale = [&](size_t dst_row, const uint16_t* Wsrc, const uint16_t* bsrc) {
+            for (int t = 0; t < W / 128; ++t) {
+                put(dst_row + (size_t)t * 256, Wsrc, bsrc, (size_t)t * 128, 128);            // shift rows
+                put(dst_row + (size_t)t * 256 + 128, Wsrc, bsrc, (size_t)W + t * 128, 128);  // scale rows
+            }
+        };
+        for (int b = 0; b < L; ++b) {
+            const uint16_t* Wm = w->Wmod + (size_t)b * 3 * W * W;
+            const uint16_t* bm = w->bmod + (size_t)b * 3 * W;
+            put_shift_scale(b * blk_rows, Wm, bm);
+            put(b * blk_rows + 2 * (size_t)W, Wm, bm, 2 * (size_t)W, W);  // gate rows
+            put(b * blk_rows + 3 * (size_t)W, w->W1 + (size_t)b * W * W, w->b1 + (size_t)b * W, 0, W);
+            put(b * blk_rows + 4 * (size_t)W, w->W2 + (size_t)b * W * W, w->b2 + (size_t)b * W, 0, W);
+        }
+        put_shift_scale(fm_row0, w->Wfm, w->bfm);
+        put(out_row0, w->Wout, w->bout, 0, C);
+        TRY(dev_alloc(H, &H->Wcat, cat_rows * W, false));
+        TRY(dev_alloc(H, &H->bias_cat, cat_rows, false));
+        TRY(upload(H->Wcat, cat.data(), cat.size() * 2));
+        TRY(upload(H->bias_cat, bias.data(), bias.size() * 4));
+    }
+    {
+        std::vector<uint16_t> win((size_t)W * XB_COLS, 0);
+        for (int o = 0; o < W; ++o) memcpy(&win[(size_t)o * XB_COLS], w->Win + (size_t)o * C, (size_t)C * 2);
+        TRY(dev_alloc(H, &H->Win, win.size(), false));
+        TRY(upload(H->Win, win.data(), win.size() * 2));
+    }
+    TRY(dev_alloc(H, &H->Wc, (size_t)W * Dc, false));
+    TRY(upload(H->Wc, w->Wc, (size_t)W * Dc * 2));
+    TRY(dev_alloc(H, &H->Wt1, (size_t)W * d.F, false));
+    TRY(upload(H->Wt1, w->Wt1, (size_t)W * d.F * 2));
+    TRY(dev_alloc(H, &H->Wt2, (size_t)W * W, false));
+    TRY(upload(H->Wt2, w->Wt2, (size_t)W * W * 2));
+    TRY(dev_alloc(H, &H->bc, W, false));
+    TRY(upload_bias(H->bc, w->bc, W));
+    TRY(dev_alloc(H, &H->bin, W, false));
+    TRY(upload_bias(H->bin, w->bin, W));
+    TRY(dev_alloc(H, &H->bt1, W, false));
+    TRY(upload_bias(H->bt1, w->bt1, W));
+    TRY(dev_alloc(H, &H->bt2, W, false));
+    TRY(upload_bias(H->bt2, w->bt2, W));
+    const int kmax = d.K_max > 0 ? d.K_max : 1;
+    TRY(dev_alloc(H, &H->temb, (size_t)kmax * W, true));
+    TRY(dev_alloc(H, &H->temb_hidden, (size_t)kmax * W, true));
+
+    // ---- scratch ----
+    TRY(dev_alloc(H, &H->z, R * Dc, true));
+    TRY(dev_alloc(H, &H->xb, R * XB_COLS, true));  // columns >= C stay zero for ever
+    TRY(dev_alloc(H, &H->s, R * W, true));
+    TRY(dev_alloc(H, &H->u, R * W, true));
+    TRY(dev_alloc(H, &H->a, R * W, true));
+    TRY(dev_alloc(H, &H->g, R * W, true));
+    TRY(dev_alloc(H, &H->x, R * C, true));
+    TRY(dev_alloc(H, &H->c, R * W, true));
+    TRY(dev_alloc(H, &H->h, R * W, true));
+    TRY(dev_alloc(H, &H->stats, R * H->NT, true));
+    TRY(dev_alloc(H, &H->counters, (size_t)H->max_tiles, true));
+    TRY(dev_alloc(H, &H->status, 2, true));
+
+    // ---- op table of one step ----
+    {
+        std::vector<StepOp> ops;
+        int cum = 0;
+        auto add = [&](int type, int ntiles, int ma, int mb, size_t b_row0, int kblocks, int umma_n, int blk) {
+            StepOp o{type, ntiles, cum, ma, mb, (int)b_row0, kblocks, umma_n, blk};
+            ops.push_back(o);
+            cum += ntiles;
+        };
+        const int NT = H->NT, kW = W / BK;
+        add(OP_IN, NT, MAP_XB, MAP_WIN, 0, 1, BN, -1);
+        for (int b = 0; b < L; ++b) {
+            add(OP_MOD, 3 * NT, MAP_S, MAP_WCAT, b * blk_rows, kW, BN, b);
+            add(OP_G1, NT, MAP_U, MAP_WCAT, b * blk_rows + 3 * (size_t)W, kW, BN, b);
+            add(OP_G2, NT, MAP_A, MAP_WCAT, b * blk_rows + 4 * (size_t)W, kW, BN, b);
+        }
+        add(OP_FMOD, 2 * NT, MAP_S, MAP_WCAT, fm_row0, kW, BN, -1);
+        add(OP_OUT, 1, MAP_U, MAP_WOUT, out_row0, kW, C, -1);
+        if (cum != H->T_step || (int)ops.size() != H->n_step_ops) {
+            free_all(H);
+            delete H;
+            return ARDIFF_ERR_UNSUPPORTED;
+        }
+        TRY(dev_alloc(H, &H->step_ops, ops.size(), false));
+        TRY(upload(H->step_ops, ops.data(), ops.size() * sizeof(StepOp)));
+    }
+    H->T_chain = H->T_pro + d.K_max * H->T_step;  // recomputed per call for the call's K
+
+    // ---- tensor maps ----
+    {
+        CUtensorMap maps[MAP_COUNT];
+        bool ok = true;
+        ok &= make_map(&maps[MAP_Z], H->z, R, Dc, BM);
+        ok &= make_map(&maps[MAP_XB], H->xb, R, XB_COLS, BM);
+        ok &= make_map(&maps[MAP_S], H->s, R, W, BM);
+        ok &= make_map(&maps[MAP_U], H->u, R, W, BM);
+        ok &= make_map(&maps[MAP_A], H->a, R, W, BM);
+        ok &= make_map(&maps[MAP_WC], H->Wc, W, Dc, BN);
+        ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, BN);
+        ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, BN);
+        ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C);
+        if (!ok) {
+            free_all(H);
+            delete H;
+            return ARDIFF_ERR_CUDA;
+        }
+        TRY(dev_alloc(H, &H->maps, MAP_COUNT, false));
+        TRY(upload(H->maps, maps, sizeof(maps)));
+    }
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        free_all(H);
+        delete H;
+        return ARDIFF_ERR_CUDA;
+    }
+    *head_out = H;
+    return ARDIFF_OK;
+}
+
+extern "C" int ardiff_head_destroy(ardiff_head* H) {
+    if (!H) return ARDIFF_OK;
+    cudaSetDevice(H->device);
+    cudaDeviceSynchronize();
+    free_all(H);
+    delete H;
+    return ARDIFF_OK;
+}
+
+extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const float* noise,
+                                  const float* t_sched, int32_t K, const int32_t* idx, const int32_t* count,
+                                  float* out, void* stream) {
+    if (!H || !idx || !count) return ARDIFF_ERR_NULL;
+    if (K < 0 || K > H->d.K_max) return ARDIFF_ERR_SHAPE;
+    if (H->d.max_tokens > 0 && (!cond || !noise || !out || !t_sched)) return ARDIFF_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(cond) & 15u) return ARDIFF_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(noise) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u))
+        return ARDIFF_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != H->device) return ARDIFF_ERR_CUDA;
+    const int W = H->d.W, C = H->d.C;
+    int launches = 0;
+
+    if (K == 0) {
+        copy_noise_rows_kernel<<<H->n_sm * 4, 256, 0, st>>>(noise, idx, count, (int)H->d.max_tokens, C, out);
+        ardiff::set_launch_count(1);
+        return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+    }
+
+    TimeArgs ta;
+    for (int k = 0; k < K; ++k) ta.t[k] = t_sched[k];
+    temb_hidden_kernel<<<dim3((W + 7) / 8, K), 256, H->d.F * sizeof(float), st>>>(H->Wt1, H->bt1, W, H->d.F, ta,
+                                                                                  H->temb_hidden);
+    temb_out_kernel<<<dim3((W + 7) / 8, K), 256, 0, st>>>(H->Wt2, H->bt2, W, H->temb_hidden, H->temb);
+    launches += 2;
+    if (cudaMemsetAsync(H->counters, 0, sizeof(int) * (size_t)H->max_tiles, st) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    if (cudaMemsetAsync(H->status + 1, 0, sizeof(int), st) != cudaSuccess) return ARDIFF_ERR_CUDA;
+
+    HeadParams P;
+    memset(&P, 0, sizeof(P));
+    P.C = C; P.Dc = H->d.Dc; P.W = W; P.L = H->d.L; P.K = K; P.NT = H->NT; P.TG = H->TG; P.slots = H->slots;
+    P.T_pro = H->T_pro; P.T_step = H->T_step; P.T_chain = H->T_pro + K * H->T_step; P.n_step_ops = H->n_step_ops;
+    P.max_tokens = (int)H->d.max_tokens;
+    P.step_ops = H->step_ops; P.maps = H->maps;
+    P.cond = reinterpret_cast<const bf16*>(cond); P.noise = noise; P.idx = idx; P.count = count; P.out = out;
+    P.z = H->z; P.xb = H->xb; P.s = H->s; P.u = H->u; P.a = H->a; P.g = H->g;
+    P.x = H->x; P.c = H->c; P.h = H->h; P.stats = H->stats;
+    P.bias_cat = H->bias_cat; P.bc = H->bc; P.bin = H->bin; P.temb = H->temb;
+    P.counters = H->counters; P.status = H->status; P.abort_flag = H->status + 1;
+    for (int k = 0; k < K; ++k) P.dt[k] = (float)((double)t_sched[k + 1] - (double)t_sched[k]);
+
+    void* args[] = {&P};
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(head_kernel), dim3(H->grid), dim3(NUM_THREADS), args,
+                                    SMEM_BYTES, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ARDIFF_ERR_CUDA;
+    }
+    launches += 1;
+    ardiff::set_launch_count(launches);
+    return ARDIFF_OK;
+}
+
+extern "C" int ardiff_head_status(ardiff_head* H, void* stream) {
+    if (!H) return ARDIFF_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    int v[2] = {0, 0};
+    if (cudaMemcpy(v, H->status, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    if (v[0] != 0 && cudaMemset(H->status, 0, sizeof(int)) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    return v[0];
+}
+
+// Internal (not part of the public header): device pointers of the head's scratch arrays, for
+// bring-up scripts that compare intermediates. name: z xb s u a g x c h temb
+extern "C" void* ardiff_head_debug_ptr(ardiff_head* H, const char* name) {
+    if (!H || !name) return nullptr;
+    if (!strcmp(name, "z")) return H->z;
+    if (!strcmp(name, "xb")) return H->xb;
+    if (!strcmp(name, "s")) return H->s;
+    if (!strcmp(name, "u")) return H->u;
+    if (!strcmp(name, "a")) return H->a;
+    if (!strcmp(name, "g")) return H->g;
+    if (!strcmp(name, "x")) return H->x;
+    if (!strcmp(name, "c")) return H->c;
+    if (!strcmp(name, "h")) return H->h;
+    if (!strcmp(name, "temb")) return H->temb;
+    if (!strcmp(name, "counters")) return H->counters;
+    return nullptr;
+}
+
+// Internal: synchronous device-to-host copy for bring-up scripts.
+extern "C" int ardiff_debug_copy_to_host(void* dst, const void* src, size_t bytes) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return ARDIFF_ERR_CUDA;
+    return cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+}

@@ -1,0 +1,204 @@
+"""GPU parity of the K-step head against the fp64 oracle, through the C ABI.
+
+Agreement bar: per token, max |out - oracle| <= 2e-2 * RMS(oracle row) (bf16 GEMM operands, fp32
+accumulation on the GPU; no rounding in the oracle). The same bar is applied to the velocity
+(out - noise) on one-step runs, where the noise no longer props up the RMS.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+import paper_2512_08537_b200 as ardiff
+from gpu_util import dev_bf16, dev_f32, require_cuda
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 2e-2
+SENTINEL = -777.0
+
+
+def make_head(wl, weights, max_tokens=None, K_max=None):
+    return ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K if K_max is None else K_max,
+                       wl.n if max_tokens is None else max_tokens, weights)
+
+
+def run_head(head, cond_bits, noise, t, idx_np, n_rows=None):
+    dev = require_cuda()
+    cond = dev_bf16(cond_bits)
+    nz = dev_f32(noise)
+    idx = torch.from_numpy(np.ascontiguousarray(idx_np, dtype=np.int32)).to(dev)
+    if idx.numel() == 0:
+        idx = torch.zeros(1, dtype=torch.int32, device=dev)
+    count = torch.tensor([len(idx_np)], dtype=torch.int32, device=dev)
+    out = torch.full(noise.shape, SENTINEL, dtype=torch.float32, device=dev)
+    head.ardiff_head_sample(cond, nz, t, idx, count, out)
+    st = head.status()
+    assert st == 0, ardiff.strerror(st)
+    return out.cpu().numpy()
+
+
+def assert_parity(got, want, rows, what="out"):
+    err = np.abs(got[rows].astype(np.float64) - want[rows]).max(axis=1)
+    rms = np.sqrt((want[rows] ** 2).mean(axis=1))
+    worst = float((err / rms).max())
+    assert worst <= REL_TOL, f"{what}: worst max|err|/rms = {worst:.3e}"
+    return worst
+
+
+def sample_tokens(idx, extra=96, seed=0):
+    """First tile, a middle tile, the last (ragged) tile, and some random survivors."""
+    S = len(idx)
+    pos = set(range(min(S, 128)))
+    pos |= set(range(max(0, (S // 256) * 128), min(S, (S // 256) * 128 + 64)))
+    pos |= set(range(max(0, S - (S % 128 or 128)), S))
+    rng = np.random.default_rng(seed)
+    pos |= set(int(p) for p in rng.integers(0, S, size=extra))
+    return np.array(sorted(pos), dtype=np.int64)
+
+
+def test_cfg1_all_tokens_gate_then_head():
+    dev = require_cuda()
+    wl = synth.workload("cfg1")
+    feat_bits = synth.features(wl)
+    H = oracle.entropy(feat_bits)
+    tau = float(np.median(H))
+    _, mask_o, idx_o, count_o = oracle.gate(feat_bits, tau)
+    w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    want = oracle.head_sample(w, cond_bits, noise, t, idx_o)
+    head = make_head(wl, w)
+    mask, idx, count, _ = ardiff.ardiff_entropy_gate(dev_bf16(feat_bits), tau)
+    out = torch.full(noise.shape, SENTINEL, dtype=torch.float32, device=dev)
+    head.ardiff_head_sample(dev_bf16(cond_bits), dev_f32(noise), t, idx, count, out)
+    assert head.status() == 0
+    got = out.cpu().numpy()
+    assert int(count.item()) == count_o
+    assert_parity(got, want, idx_o)
+    dropped = np.flatnonzero(mask_o == 0)
+    assert np.all(got[dropped] == SENTINEL)          # rows of filtered tokens are never written
+    head.close()
+
+
+@pytest.mark.parametrize("std", [0.02, None])
+@pytest.mark.parametrize("count", [1, 64, 127, 128, 129, 300])
+def test_small_head_ragged_counts(std, count):
+    wl = synth.workload("cfg1", n=320)
+    w, cond_bits, noise, t = synth.head_weights(wl, std=std), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    idx = np.random.default_rng(count).permutation(wl.n)[:count].astype(np.int32)   # any order
+    want = oracle.head_sample(w, cond_bits, noise, t, idx)
+    head = make_head(wl, w)
+    got = run_head(head, cond_bits, noise, t, idx)
+    assert_parity(got, want, idx)
+    rest = np.setdiff1d(np.arange(wl.n), idx)
+    assert np.all(got[rest] == SENTINEL)
+    head.close()
+
+
+@pytest.mark.parametrize("std", [0.02, None])
+def test_velocity_parity_one_step(std):
+    wl = synth.workload("cfg1", n=256, K=1)
+    w, cond_bits, noise, t = synth.head_weights(wl, std=std), synth.cond(wl), synth.noise(wl), synth.t_sched(1)
+    idx = np.arange(wl.n, dtype=np.int32)
+    want = oracle.head_sample(w, cond_bits, noise, t, idx)
+    head = make_head(wl, w)
+    got = run_head(head, cond_bits, noise, t, idx)
+    assert_parity(got - noise, want - noise, idx, "velocity")
+    head.close()
+
+
+def test_k0_copies_noise_and_count0_writes_nothing():
+    wl = synth.workload("cfg1", n=200)
+    w, cond_bits, noise = synth.head_weights(wl), synth.cond(wl), synth.noise(wl)
+    head = make_head(wl, w)
+    idx = np.arange(0, 200, 3, dtype=np.int32)
+    got = run_head(head, cond_bits, noise, synth.t_sched(0), idx)
+    assert np.array_equal(got[idx], noise[idx])
+    assert np.all(got[np.setdiff1d(np.arange(200), idx)] == SENTINEL)
+    got0 = run_head(head, cond_bits, noise, synth.t_sched(4), np.zeros(0, np.int32))
+    assert np.all(got0 == SENTINEL)
+    head.close()
+
+
+def test_nonuniform_schedule_and_k_sweep():
+    wl = synth.workload("cfg1", n=192, K=8)
+    w, cond_bits, noise = synth.head_weights(wl, std=None), synth.cond(wl), synth.noise(wl)
+    head = make_head(wl, w, K_max=8)
+    idx = np.arange(wl.n, dtype=np.int32)
+    for K in (1, 2, 3, 8):
+        t = np.sort(np.random.default_rng(K).uniform(0.0, 1.0, size=K + 1)).astype(np.float32)
+        want = oracle.head_sample(w, cond_bits, noise, t, idx)
+        got = run_head(head, cond_bits, noise, t, idx)
+        assert_parity(got, want, idx, f"K={K}")
+    # reversed time direction
+    t = np.array([1.0, 0.5, 0.0], np.float32)
+    assert_parity(run_head(head, cond_bits, noise, t, idx), oracle.head_sample(w, cond_bits, noise, t, idx), idx)
+    head.close()
+
+
+def test_two_calls_on_one_head_give_identical_results():
+    wl = synth.workload("cfg1", n=300)
+    w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    head = make_head(wl, w)
+    idx = np.arange(wl.n, dtype=np.int32)
+    a = run_head(head, cond_bits, noise, t, idx)
+    b = run_head(head, cond_bits, noise, t, idx)
+    assert np.array_equal(a, b)
+    head.close()
+
+
+@pytest.mark.parametrize("name,extra", [("cfg2", 160), ("cfg3", 48), ("cfg4", 32)])
+def test_workload_configs_sampled_tokens(name, extra):
+    """Full-size gate -> head run; the oracle checks the first, a middle and the last (ragged)
+    token tile plus random survivors one by one (tokens are independent)."""
+    dev = require_cuda()
+    wl = synth.workload(name)
+    feat_bits = synth.features(wl)
+    H = oracle.entropy(feat_bits)
+    Hs = np.sort(H)
+    k = int(round(wl.filter_q * wl.n))
+    tau = 0.5 * (Hs[k - 1] + Hs[k])
+    w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    head = make_head(wl, w)
+    mask, idx, count, _ = ardiff.ardiff_entropy_gate(dev_bf16(feat_bits), tau)
+    out = torch.full(noise.shape, SENTINEL, dtype=torch.float32, device=dev)
+    head.ardiff_head_sample(dev_bf16(cond_bits), dev_f32(noise), t, idx, count, out)
+    assert head.status() == 0
+    S = int(count.item())
+    idx_h = idx.cpu().numpy()[:S]
+    got = out.cpu().numpy()
+    if name != "cfg2":                      # keep the oracle's share of the run to seconds
+        pos = sample_tokens(idx_h, extra=extra)
+        pos = np.concatenate([pos[:16], pos[len(pos) // 2: len(pos) // 2 + 8], pos[-16:],
+                              np.random.default_rng(1).choice(pos, size=extra, replace=False)])
+        pos = np.unique(pos)
+    else:
+        pos = sample_tokens(idx_h, extra=extra)
+    toks = idx_h[pos]
+    want = oracle.head_sample(w, cond_bits, noise, t, toks)
+    assert_parity(got, want, toks, name)
+    # properties that hold for every token: written iff kept, finite
+    kept = np.zeros(wl.n, bool)
+    kept[idx_h] = True
+    assert np.all(got[~kept] == SENTINEL)
+    assert np.all(np.isfinite(got[kept])) and not np.any(got[kept] == SENTINEL)
+    head.close()
+
+
+def test_bad_arguments_are_rejected():
+    require_cuda()
+    wl = synth.workload("cfg1")
+    w = synth.head_weights(wl)
+    with pytest.raises(ardiff.ArdiffError):
+        ardiff.Head(wl.C, wl.Dc, 250, wl.L, wl.F, 4, 64, w)          # W not a multiple of 256
+    with pytest.raises(ardiff.ArdiffError):
+        ardiff.Head(8, wl.Dc, wl.W, wl.L, wl.F, 4, 64, w)            # C too small
+    head = make_head(wl, w)
+    lib = ardiff.lib()
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    p = buf.data_ptr()
+    t = synth.t_sched(4)
+    assert lib.ardiff_head_sample(head._h, p, p, t.ctypes.data, 5, p, p, p, None) == ardiff.ARDIFF_ERR_SHAPE
+    assert lib.ardiff_head_sample(head._h, p, p, t.ctypes.data, 4, None, p, p, None) == ardiff.ARDIFF_ERR_NULL
+    assert lib.ardiff_head_sample(head._h, p + 2, p, t.ctypes.data, 4, p, p, p, None) == ardiff.ARDIFF_ERR_ALIGN
+    head.close()
