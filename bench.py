@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark of the entropy-gated K-step head hot path (gate -> compaction -> head).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+One step = one pass of the whole path over one batch of synthetic draft tokens. Prints one JSON
+line: gated draft tokens/s (device-resident inputs), the same through the host-buffer C-ABI call
+(`e2e`), the roofline of the dominant kernel (the persistent head kernel, tensor-bound), the gate's
+HBM figure, clocks sampled during the timed region, and the fp64 CPU oracle timed on a bounded
+sample (`cpu_baseline`). `--impl reference` times only that oracle.
+With N > 1 (torchrun) every rank runs the same batch shape on its own GPU: no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+METRIC = "gated draft tokens/sec through K-step head"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 512 << 20
+# dram bytes per launch of the head kernel from the ncu capture summarised under profiles/
+TRAFFIC_BYTES = {}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def quantile_tau(H: np.ndarray, q: float) -> float:
+    Hs = np.sort(H[~np.isnan(H)])
+    k = int(round(q * len(Hs)))
+    if k <= 0:
+        return -1.0
+    if k >= len(Hs):
+        return float(Hs[-1]) + 1.0
+    return 0.5 * (float(Hs[k - 1]) + float(Hs[k]))
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places that touch oracle/)
+# ----------------------------------------------------------------------------------------------
+def oracle_step(wl, weights, m):
+    """Oracle gate + head on the first m draft tokens; returns (seconds, kept)."""
+    import oracle
+    feat = synth.features(wl, 0, m)
+    cond, noise, t = synth.cond(wl, 0, m), synth.noise(wl, 0, m), synth.t_sched(wl.K)
+    H = oracle.entropy(feat)
+    tau = quantile_tau(H, wl.filter_q)
+    t0 = time.perf_counter()
+    _, _, idx, count = oracle.gate(feat, tau)
+    oracle.head_sample(weights, cond, noise, t, idx)
+    return time.perf_counter() - t0, count
+
+
+def cpu_baseline(wl, weights, m):
+    import oracle
+    oracle.build()
+    sec, kept = oracle_step(wl, weights, m)
+    return {"value": m / sec, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"first {m} draft tokens of {wl.name} ({kept} kept), gate + {wl.K}-step head, "
+                      f"fp64, {sec:.2f} s"}
+
+
+def run_reference(args, wl):
+    """--impl reference: the fp64 oracle, as it stands, on this machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    weights = synth.head_weights(wl)
+    m = args.ref_tokens
+    for _ in range(args.warmup):
+        oracle_step(wl, weights, m)
+    secs = []
+    for _ in range(args.steps):
+        s, kept = oracle_step(wl, weights, m)
+        secs.append(s)
+    per = sum(secs) / len(secs)
+    val = m / per
+    sample = f"each step: first {m} draft tokens of {wl.name} ({kept} kept), gate + {wl.K}-step head, fp64"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "sample_tokens": m},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU during the timed region (read-only NVML)."""
+
+    def __init__(self, dev_index: int, period_s: float = 0.005):
+        import threading
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = dev_index
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if dev_index < len(ids) and ids[dev_index].isdigit():
+                    phys = int(ids[dev_index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+            return
+        self.period = period_s
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+                 "hw_thermal_slowdown": 0x40}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for nm, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(nm)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def upload_bf16(torch, bits, dev):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+
+
+def run_gpu(args, wl):
+    import torch
+    import paper_2512_08537_b200 as ardiff
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    ardiff.lib()  # fails loudly when libardiff.so cannot be loaded
+
+    # ---- inputs: seeded on the host, resident in HBM before the timed region ----
+    wl_r = synth.workload(wl.name, seed=wl.seed + 1000 * rank) if world > 1 else wl
+    weights = synth.head_weights(wl)
+    n = wl.n
+    feat = torch.empty((n, wl.d), dtype=torch.bfloat16, device=dev)
+    slab = 32768
+    for r0 in range(0, n, slab):
+        feat[r0:r0 + slab] = upload_bf16(torch, synth.features(wl_r, r0, min(slab, n - r0)), dev)
+    cond_h, noise_h = synth.cond(wl_r), synth.noise(wl_r)
+    cond = upload_bf16(torch, cond_h, dev)
+    noise = torch.from_numpy(noise_h).to(dev)
+    t = synth.t_sched(wl.K)
+    head = ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K, n, weights)
+    head.set_timing(True)
+    mask = torch.empty(n, dtype=torch.uint8, device=dev)
+    idx = torch.empty(n, dtype=torch.int32, device=dev)
+    count = torch.zeros(1, dtype=torch.int32, device=dev)
+    ent = torch.empty(n, dtype=torch.float32, device=dev)
+    out = torch.zeros((n, wl.C), dtype=torch.float32, device=dev)
+    # tau: the quantile of the gate's own entropies that drops filter_q of the tokens (set-up, untimed)
+    ardiff.ardiff_entropy_gate(feat, -1.0, mask, idx, count, ent)
+    torch.cuda.synchronize()
+    tau = quantile_tau(ent.cpu().numpy().astype(np.float64), wl.filter_q)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ardiff.ardiff_entropy_gate(feat, tau, mask, idx, count, stream=stream)
+        l1 = ardiff.last_launch_count()
+        head.ardiff_head_sample(cond, noise, t, idx, count, out, stream=stream)
+        return l1 + ardiff.last_launch_count()
+
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    if head.status() != 0:
+        raise RuntimeError("head kernel reported a device-side timeout")
+    S = int(count.item())
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    head_ms, launches = [], 0
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    for i in range(args.steps):
+        flush.fill_(i & 0xff)                     # L2 flush between timed iterations (not timed)
+        ev[i][0].record(stream)
+        ardiff.ardiff_entropy_gate(feat, tau, mask, idx, count, stream=stream)
+        launches += ardiff.last_launch_count()
+        ev[i][1].record(stream)
+        head.ardiff_head_sample(cond, noise, t, idx, count, out, stream=stream)
+        launches += ardiff.last_launch_count()
+        ev[i][2].record(stream)
+        head_ms.append(head.last_kernel_ms())     # waits for this step's head kernel
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop() if sampler else None
+    gate_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    step_ms = [e[0].elapsed_time(e[2]) for e in ev]
+    total_ms = sum(step_ms)
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    if head.status() != 0:
+        raise RuntimeError("head kernel reported a device-side timeout")
+    ms_per_step = total_ms / args.steps
+    value = world * n / (ms_per_step * 1e-3)
+
+    # ---- e2e: the host-buffer C-ABI call; host<->device copies inside the timed region ----
+    pipe = ardiff.Pipeline(head, n, wl.d)
+    feat_pin = torch.empty((n, wl.d), dtype=torch.bfloat16).pin_memory()
+    feat_pin.copy_(feat)
+    cond_pin = torch.from_numpy(cond_h.view(np.int16)).view(torch.bfloat16).pin_memory()
+    noise_pin = torch.from_numpy(noise_h).pin_memory()
+    out_pin = torch.empty((n, wl.C), dtype=torch.float32).pin_memory()
+    mask_pin = torch.empty(n, dtype=torch.uint8).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        pipe.ardiff_pipeline_run_host(feat_pin, cond_pin, noise_pin, tau, t, out_pin, mask_pin, stream=stream)
+    if dist is not None:
+        dist.barrier()
+    e2e_ms = []
+    for _ in range(e2e_steps):
+        flush.fill_(3)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        kept = pipe.ardiff_pipeline_run_host(feat_pin, cond_pin, noise_pin, tau, t, out_pin, mask_pin, stream=stream)
+        e1.record(stream)
+        e1.synchronize()
+        e2e_ms.append(e0.elapsed_time(e1))
+    e2e_total = sum(e2e_ms)
+    if dist is not None:
+        tt = torch.tensor([e2e_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_total = float(tt.item())
+    e2e_value = world * n / (e2e_total / e2e_steps * 1e-3)
+    h2d = n * (2 * wl.d + 2 * wl.Dc + 4 * wl.C)
+    d2h = n * (4 * wl.C + 1) + 4
+    pipe.close()
+
+    if rank == 0:
+        pk = peaks()
+        hk_ms = statistics.mean(head_ms)
+        flops = S * wl.flops_per_token()
+        achieved = flops / (hk_ms * 1e-3) / 1e12
+        g_ms = statistics.mean(gate_ms)
+        gate_gbs = wl.gate_bytes() / (g_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "tokens_per_gpu": n, "survivors": S, "d": wl.d, "C": wl.C,
+                       "Dc": wl.Dc, "W": wl.W, "L": wl.L, "K": wl.K, "tau": tau,
+                       "l2": "512 MiB written between timed iterations", "parallelism": f"dp{world}"},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": achieved / pk["bf16_tflops"], "traffic": TRAFFIC_BYTES.get(wl.name),
+                         "kernel": "head_kernel", "peak_source": f"{pk['source']} burst bf16",
+                         "kernel_ms": hk_ms, "flops_per_launch": flops},
+            "gate": {"bound": "hbm", "achieved": gate_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": gate_gbs / pk["hbm_gbs"], "ms": g_ms, "note": "gate + compaction launches"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_total / e2e_steps, "steps": e2e_steps},
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl, weights, args.cpu_tokens)
+        print(json.dumps(line), flush=True)
+    head.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--K", type=int, default=None, help="override the number of sampler steps")
+    ap.add_argument("--filter", type=float, default=None, help="override the fraction of tokens dropped")
+    ap.add_argument("--cpu-tokens", type=int, default=6144, help="draft tokens of the cpu_baseline sample")
+    ap.add_argument("--ref-tokens", type=int, default=256, help="draft tokens per --impl reference step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    over = {}
+    if args.K is not None:
+        over["K"] = args.K
+    if args.filter is not None:
+        over["filter_q"] = args.filter
+    wl = synth.workload(args.workload, **over)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_gpu(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -152,6 +152,31 @@ int ardiff_head_sample(const ardiff_head* head, const void* cond, const float* n
  * ARDIFF_ERR_SHAPE if *count exceeded max_tokens. Clears it. */
 int ardiff_head_status(ardiff_head* head, void* stream);
 
+/* Profiling aid: with on != 0, every later ardiff_head_sample on this head records CUDA events
+ * on its stream directly around the persistent head kernel. ardiff_head_last_kernel_ms waits
+ * for that kernel and writes its device time in milliseconds (ERR_SHAPE if nothing was timed). */
+int ardiff_head_set_timing(ardiff_head* head, int on);
+int ardiff_head_last_kernel_ms(ardiff_head* head, float* ms);
+
+/* ---------------------------------------------------------------------------------------
+ * Host-buffer front end: one call takes a batch that lives in HOST memory through the whole
+ * path (copy in, gate, head, copy out). The pipeline object owns device staging buffers for
+ * up to max_n tokens of feature width d, conditioning width Dc and token dim C (which must
+ * match the head's). Pinned host buffers make the copies asynchronous; pageable ones work too.
+ *
+ *   feat   host bf16 [n][d],  cond host bf16 [n][Dc],  noise host float [n][C]
+ *   out    host float [n][C]: rows of kept tokens hold the sample, dropped rows are 0
+ *   mask   host uint8 [n],    count host int32 [1]
+ * The call waits for `stream` before it returns, so the host outputs are valid on return.
+ * ------------------------------------------------------------------------------------- */
+typedef struct ardiff_pipeline ardiff_pipeline;
+int ardiff_pipeline_create(ardiff_head* head, int64_t max_n, int32_t d, int32_t Dc, int32_t C,
+                           ardiff_pipeline** pipeline_out);
+int ardiff_pipeline_destroy(ardiff_pipeline* pipeline);
+int ardiff_pipeline_run_host(ardiff_pipeline* pipeline, const void* feat, const void* cond,
+                             const float* noise, int64_t n, float tau, const float* t_sched, int32_t K,
+                             float* out, uint8_t* mask, int32_t* count, void* stream);
+
 /* Number of kernel launches the last ardiff_head_sample / ardiff_entropy_gate call on this
  * thread enqueued (for launch accounting by benchmarks). */
 int ardiff_last_launch_count(void);

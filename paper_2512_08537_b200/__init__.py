@@ -65,6 +65,16 @@ def lib() -> ctypes.CDLL:
             L.ardiff_head_sample.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
             L.ardiff_head_status.restype = ctypes.c_int
             L.ardiff_head_status.argtypes = [vp, vp]
+            L.ardiff_head_set_timing.restype = ctypes.c_int
+            L.ardiff_head_set_timing.argtypes = [vp, ctypes.c_int]
+            L.ardiff_head_last_kernel_ms.restype = ctypes.c_int
+            L.ardiff_head_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+            L.ardiff_pipeline_create.restype = ctypes.c_int
+            L.ardiff_pipeline_create.argtypes = [vp, i64, i32, i32, i32, ctypes.POINTER(vp)]
+            L.ardiff_pipeline_destroy.restype = ctypes.c_int
+            L.ardiff_pipeline_destroy.argtypes = [vp]
+            L.ardiff_pipeline_run_host.restype = ctypes.c_int
+            L.ardiff_pipeline_run_host.argtypes = [vp, vp, vp, vp, i64, f32, vp, i32, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -159,10 +169,54 @@ class Head:
     def status(self, stream=None) -> int:
         return int(lib().ardiff_head_status(self._h, _stream_ptr(stream)))
 
+    def set_timing(self, on: bool):
+        _check(lib().ardiff_head_set_timing(self._h, 1 if on else 0), "ardiff_head_set_timing")
+
+    def last_kernel_ms(self) -> float:
+        ms = ctypes.c_float(0.0)
+        _check(lib().ardiff_head_last_kernel_ms(self._h, ctypes.byref(ms)), "ardiff_head_last_kernel_ms")
+        return float(ms.value)
+
     def close(self):
         if getattr(self, "_h", None) is not None and self._h:
             lib().ardiff_head_destroy(self._h)
             self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Pipeline:
+    """Host-buffer front end (ardiff_pipeline_*): device staging for up to max_n tokens."""
+
+    def __init__(self, head: Head, max_n: int, d: int):
+        self.head = head
+        self.d, self.Dc, self.C = d, head.desc.Dc, head.desc.C
+        p = ctypes.c_void_p()
+        _check(lib().ardiff_pipeline_create(head._h, max_n, d, self.Dc, self.C, ctypes.byref(p)),
+               "ardiff_pipeline_create")
+        self._p = p
+
+    def ardiff_pipeline_run_host(self, feat, cond, noise, tau, t_sched, out, mask, stream=None) -> int:
+        """feat/cond: host bf16 tensors, noise/out: host f32, mask: host u8 (pinned or not).
+        Returns the number of kept tokens. Synchronises the stream."""
+        import numpy as np
+        ts = np.ascontiguousarray(t_sched, dtype=np.float32)
+        n = feat.shape[0]
+        count = ctypes.c_int32(0)
+        rc = lib().ardiff_pipeline_run_host(self._p, feat.data_ptr(), cond.data_ptr(), noise.data_ptr(), n,
+                                            float(tau), ts.ctypes.data, ts.shape[0] - 1, out.data_ptr(),
+                                            mask.data_ptr(), ctypes.addressof(count), _stream_ptr(stream))
+        _check(rc, "ardiff_pipeline_run_host")
+        return int(count.value)
+
+    def close(self):
+        if getattr(self, "_p", None) is not None and self._p:
+            lib().ardiff_pipeline_destroy(self._p)
+            self._p = None
 
     def __del__(self):
         try:

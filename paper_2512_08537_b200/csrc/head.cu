@@ -779,6 +779,9 @@ struct ardiff_head {
     int *counters, *status;  // status[0] = status word, status[1] = abort flag
     StepOp* step_ops;
     CUtensorMap* maps;
+    // optional timing of the persistent kernel
+    int timing, timed;
+    cudaEvent_t ev0, ev1;
 };
 
 namespace {
@@ -1018,6 +1021,8 @@ extern "C" int ardiff_head_destroy(ardiff_head* H) {
     if (!H) return ARDIFF_OK;
     cudaSetDevice(H->device);
     cudaDeviceSynchronize();
+    if (H->ev0) cudaEventDestroy(H->ev0);
+    if (H->ev1) cudaEventDestroy(H->ev1);
     free_all(H);
     delete H;
     return ARDIFF_OK;
@@ -1067,14 +1072,37 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
     for (int k = 0; k < K; ++k) P.dt[k] = (float)((double)t_sched[k + 1] - (double)t_sched[k]);
 
     void* args[] = {&P};
+    ardiff_head* Hm = const_cast<ardiff_head*>(H);
+    if (H->timing) cudaEventRecord(H->ev0, st);
     if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(head_kernel), dim3(H->grid), dim3(NUM_THREADS), args,
                                     SMEM_BYTES, st) != cudaSuccess) {
         (void)cudaGetLastError();
         return ARDIFF_ERR_CUDA;
     }
+    if (H->timing) {
+        cudaEventRecord(H->ev1, st);
+        Hm->timed = 1;
+    }
     launches += 1;
     ardiff::set_launch_count(launches);
     return ARDIFF_OK;
+}
+
+extern "C" int ardiff_head_set_timing(ardiff_head* H, int on) {
+    if (!H) return ARDIFF_ERR_NULL;
+    if (on && !H->ev0) {
+        if (cudaEventCreate(&H->ev0) != cudaSuccess || cudaEventCreate(&H->ev1) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    }
+    H->timing = on ? 1 : 0;
+    H->timed = 0;
+    return ARDIFF_OK;
+}
+
+extern "C" int ardiff_head_last_kernel_ms(ardiff_head* H, float* ms) {
+    if (!H || !ms) return ARDIFF_ERR_NULL;
+    if (!H->timed) return ARDIFF_ERR_SHAPE;
+    if (cudaEventSynchronize(H->ev1) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    return cudaEventElapsedTime(ms, H->ev0, H->ev1) == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
 }
 
 extern "C" int ardiff_head_status(ardiff_head* H, void* stream) {
