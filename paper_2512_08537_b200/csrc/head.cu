@@ -35,20 +35,31 @@ using bf16 = __nv_bfloat16;
 constexpr int BM = 128;           // tokens per tile
 constexpr int BN = 256;           // output columns per tile (UMMA N)
 constexpr int BK = 64;            // K slice per pipeline stage (128 bytes of bf16: one swizzle row)
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+// epilogue staging: every epilogue warp owns EPI_NB buffers, each one fp32 slab (32 rows x 128 B,
+// 128-byte swizzle) plus one bf16 slab (32 rows x 64 B, 64-byte swizzle), filled and drained by TMA
+constexpr int EPI_NB = 3;
+constexpr int SLAB_F = 32 * 128;
+constexpr int SLAB_H = 32 * 64;
+constexpr int EPI_BUF = SLAB_F + SLAB_H;
+constexpr int EPI_BYTES = 4 * EPI_NB * EPI_BUF;
+constexpr int NUM_BARS = 2 * STAGES + 5 + 4 * EPI_NB;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*align slack*/ + 8 * NUM_BARS + 16;
 constexpr int NUM_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
-constexpr int EPI_THREADS = 128;
 constexpr int XB_COLS = 64;       // x is fed to the in-projection as bf16, K padded to one slice
 constexpr int KMAX = 64;
 constexpr uint64_t kWaitLimitNs = 4000000000ull;   // a bounded wait gives up after 4 s
 constexpr uint64_t kDrainLimitNs = 200000000ull;   // waits for own copies in flight at exit
 
 enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_MOD, OP_G1, OP_G2, OP_FMOD, OP_OUT };
-enum MapId : int { MAP_Z = 0, MAP_XB, MAP_S, MAP_U, MAP_A, MAP_WC, MAP_WIN, MAP_WCAT, MAP_WOUT, MAP_COUNT };
+enum MapId : int {
+    MAP_Z = 0, MAP_XB, MAP_S, MAP_U, MAP_A, MAP_WC, MAP_WIN, MAP_WCAT, MAP_WOUT,   // GEMM operands
+    EMAP_H, EMAP_C, EMAP_S, EMAP_U, EMAP_A, EMAP_G,                                 // epilogue slabs
+    MAP_COUNT
+};
 
 struct StepOp {
     int type;      // OpType
@@ -199,8 +210,11 @@ __device__ __forceinline__ void decode_item(const HeadParams& P, int MT, long lo
 }
 
 // ------------------------------------------------------------------------------------------
-// epilogues. Thread `row` (0..127) of the tile owns TMEM lane `row`; `tacc` addresses its lane
-// at column 0 of the accumulator. Each handles 32 columns per tcgen05.ld.
+// epilogues. Lane r of an epilogue warp owns row r of the warp's 32-row quarter of the tile (TMEM
+// lane quarter*32 + r). Work goes in chunks of 32 accumulator columns: the chunk's global inputs
+// (h, c: fp32 slab; g: bf16 slab) arrive by TMA in a swizzled shared-memory buffer, the lane reads
+// its own row, combines it with the accumulator chunk, writes the results back into the buffer
+// (in place) and lane 0 hands the buffer to a TMA store. Loads run two chunks ahead.
 // ------------------------------------------------------------------------------------------
 struct Stats {
     float p, sd, sq;
@@ -213,6 +227,50 @@ struct Stats {
         return make_float2(mean, m2);
     }
 };
+
+struct EpiIO {            // what one item's epilogue moves per 32-column chunk (-1: nothing)
+    int nch;              // chunks
+    int ldF, ldF_col;     // fp32 slab load: map id, first column
+    int ldH, ldH_col;     // bf16 slab load
+    int stF, stF_col;     // fp32 slab store
+    int stH, stH_col;     // bf16 slab store
+};
+
+__device__ __forceinline__ EpiIO epi_io(const HeadParams& P, const Item& it) {
+    EpiIO io{BN / 32, -1, 0, -1, 0, -1, 0, -1, 0};
+    const int col0 = it.nt * BN;
+    switch (it.type) {
+        case OP_COND: io.stF = EMAP_C; io.stF_col = col0; break;
+        case OP_IN:
+            io.ldF = EMAP_C; io.ldF_col = col0; io.stF = EMAP_H; io.stF_col = col0;
+            io.stH = EMAP_S; io.stH_col = col0;
+            break;
+        case OP_MOD:
+            if (it.nt < P.W / 128) {
+                io.nch = 4; io.ldF = EMAP_H; io.ldF_col = it.nt * 128; io.stH = EMAP_U; io.stH_col = it.nt * 128;
+            } else {
+                io.stH = EMAP_G; io.stH_col = (it.nt - P.W / 128) * BN;
+            }
+            break;
+        case OP_FMOD:
+            io.nch = 4; io.ldF = EMAP_H; io.ldF_col = it.nt * 128; io.stH = EMAP_U; io.stH_col = it.nt * 128;
+            break;
+        case OP_G1: io.stH = EMAP_A; io.stH_col = col0; break;
+        case OP_G2:
+            io.ldF = EMAP_H; io.ldF_col = col0; io.ldH = EMAP_G; io.ldH_col = col0;
+            io.stF = EMAP_H; io.stF_col = col0;
+            break;
+        default: io.nch = 0; break;   // OP_OUT: register path
+    }
+    return io;
+}
+
+__device__ __forceinline__ uint32_t slabF_addr(uint32_t base, int r, int c16) {
+    return base + r * 128 + ((c16 ^ (r & 7)) << 4);
+}
+__device__ __forceinline__ uint32_t slabH_addr(uint32_t base, int r, int c16) {
+    return base + r * 64 + ((c16 ^ ((r >> 1) & 3)) << 4);
+}
 
 __device__ __forceinline__ void load_acc32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
@@ -230,78 +288,38 @@ __device__ __forceinline__ void add_bias32(float (&v)[32], const float* __restri
     }
 }
 
-__device__ __forceinline__ void store_bf16_32(bf16* dst, const float (&v)[32]) {
+__device__ __forceinline__ void slabF_read(uint32_t base, int r, float (&v)[32]) {
 #pragma unroll
-    for (int i = 0; i < 32; i += 8) {
+    for (int c = 0; c < 8; ++c) {
+        const uint4 w = ptx::lds_u4(slabF_addr(base, r, c));
+        v[4 * c] = __uint_as_float(w.x); v[4 * c + 1] = __uint_as_float(w.y);
+        v[4 * c + 2] = __uint_as_float(w.z); v[4 * c + 3] = __uint_as_float(w.w);
+    }
+}
+__device__ __forceinline__ void slabF_write(uint32_t base, int r, const float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        ptx::sts_u4(slabF_addr(base, r, c), make_uint4(__float_as_uint(v[4 * c]), __float_as_uint(v[4 * c + 1]),
+                                                       __float_as_uint(v[4 * c + 2]), __float_as_uint(v[4 * c + 3])));
+}
+__device__ __forceinline__ void slabH_read(uint32_t base, int r, float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint4 w = ptx::lds_u4(slabH_addr(base, r, c));
+        v[8 * c] = bf16lo(w.x); v[8 * c + 1] = bf16hi(w.x); v[8 * c + 2] = bf16lo(w.y); v[8 * c + 3] = bf16hi(w.y);
+        v[8 * c + 4] = bf16lo(w.z); v[8 * c + 5] = bf16hi(w.z); v[8 * c + 6] = bf16lo(w.w); v[8 * c + 7] = bf16hi(w.w);
+    }
+}
+__device__ __forceinline__ void slabH_write(uint32_t base, int r, const float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
         uint4 w;
-        w.x = pack_bf16x2(v[i], v[i + 1]);
-        w.y = pack_bf16x2(v[i + 2], v[i + 3]);
-        w.z = pack_bf16x2(v[i + 4], v[i + 5]);
-        w.w = pack_bf16x2(v[i + 6], v[i + 7]);
-        ptx::st_u4(dst + i, w);
+        w.x = pack_bf16x2(v[8 * c], v[8 * c + 1]);
+        w.y = pack_bf16x2(v[8 * c + 2], v[8 * c + 3]);
+        w.z = pack_bf16x2(v[8 * c + 4], v[8 * c + 5]);
+        w.w = pack_bf16x2(v[8 * c + 6], v[8 * c + 7]);
+        ptx::sts_u4(slabH_addr(base, r, c), w);
     }
-}
-
-__device__ __forceinline__ void store_f32_32(float* dst, const float (&v)[32]) {
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) ptx::st_f4(dst + i, make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
-}
-
-__device__ __forceinline__ void load_f32_32(const float* src, float (&v)[32]) {
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        const float4 t = ptx::ldcg_f4(src + i);
-        v[i] = t.x; v[i + 1] = t.y; v[i + 2] = t.z; v[i + 3] = t.w;
-    }
-}
-
-__device__ __forceinline__ void load_bf16_32(const bf16* src, float (&v)[32]) {
-#pragma unroll
-    for (int i = 0; i < 32; i += 8) {
-        const uint4 w = ptx::ldcg_u4(src + i);
-        v[i] = bf16lo(w.x); v[i + 1] = bf16hi(w.x); v[i + 2] = bf16lo(w.y); v[i + 3] = bf16hi(w.y);
-        v[i + 4] = bf16lo(w.z); v[i + 5] = bf16hi(w.z); v[i + 6] = bf16lo(w.w); v[i + 7] = bf16hi(w.w);
-    }
-}
-
-// c = acc + bc
-__device__ __forceinline__ void epi_cond(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
-    const int col0 = it.nt * BN;
-    float* crow = P.c + (size_t)grow * P.W + col0;
-#pragma unroll 1
-    for (int cc = 0; cc < BN / 32; ++cc) {
-        float v[32];
-        load_acc32(tacc + cc * 32, v);
-        add_bias32(v, P.bc + col0 + cc * 32);
-        store_f32_32(crow + cc * 32, v);
-    }
-}
-
-// h = acc + bin ; LN partial statistics ; s = SiLU(c + temb_k)
-__device__ __forceinline__ void epi_in(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
-    const int col0 = it.nt * BN;
-    float* hrow = P.h + (size_t)grow * P.W + col0;
-    const float* crow = P.c + (size_t)grow * P.W + col0;
-    bf16* srow = P.s + (size_t)grow * P.W + col0;
-    const float* temb = P.temb + (size_t)it.k * P.W + col0;
-    Stats st;
-#pragma unroll 1
-    for (int cc = 0; cc < BN / 32; ++cc) {
-        float v[32];
-        load_acc32(tacc + cc * 32, v);
-        add_bias32(v, P.bin + col0 + cc * 32);
-        if (cc == 0) st.init(v[0]);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) st.add(v[i]);
-        store_f32_32(hrow + cc * 32, v);
-        float cv[32];
-        load_f32_32(crow + cc * 32, cv);
-        add_bias32(cv, temb + cc * 32);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) cv[i] = silu_f(cv[i]);
-        store_bf16_32(srow + cc * 32, cv);
-    }
-    P.stats[(size_t)grow * P.NT + it.nt] = st.finish(BN);
 }
 
 __device__ __forceinline__ void row_mean_rstd(const HeadParams& P, int grow, float& mean, float& rstd) {
@@ -318,81 +336,76 @@ __device__ __forceinline__ void row_mean_rstd(const HeadParams& P, int grow, flo
     rstd = rsqrtf(m2 / (float)P.W + 1e-6f);
 }
 
-// shift/scale tile: accumulator columns [0,128) = shift, [128,256) = scale of h columns
-// [nt*128, nt*128+128):  u = LN(h) * (1 + scale) + shift
-__device__ __forceinline__ void epi_mod_ss(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
-    float mean, rstd;
-    row_mean_rstd(P, grow, mean, rstd);
-    const int hcol0 = it.nt * 128;
-    const float* hrow = P.h + (size_t)grow * P.W + hcol0;
-    bf16* urow = P.u + (size_t)grow * P.W + hcol0;
-    const float* bias = P.bias_cat + it.b_row;
-#pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
-        float sh[32], sc[32], hv[32];
-        load_acc32(tacc + cc * 32, sh);
-        load_acc32(tacc + 128 + cc * 32, sc);
-        add_bias32(sh, bias + cc * 32);
-        add_bias32(sc, bias + 128 + cc * 32);
-        load_f32_32(hrow + cc * 32, hv);
+// One 32-column chunk of one item. bufF / bufH: this warp's slabs for the chunk; r: lane.
+__device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, int cc, uint32_t tacc,
+                                          uint32_t bufF, uint32_t bufH, int r, Stats& st, float mean,
+                                          float rstd) {
+    float v[32];
+    switch (it.type) {
+        case OP_COND: {                       // c = acc + bc
+            load_acc32(tacc + cc * 32, v);
+            add_bias32(v, P.bc + it.nt * BN + cc * 32);
+            slabF_write(bufF, r, v);
+            break;
+        }
+        case OP_IN: {                         // h = acc + bin ; s = SiLU(c + temb_k)
+            load_acc32(tacc + cc * 32, v);
+            add_bias32(v, P.bin + it.nt * BN + cc * 32);
+            if (cc == 0) st.init(v[0]);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], sh[i]);
-        store_bf16_32(urow + cc * 32, hv);
-    }
-}
-
-// gate tile: g = acc + bias (columns [ (nt - W/128)*256, +256 ) of the block's gate)
-__device__ __forceinline__ void epi_mod_g(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
-    const int col0 = (it.nt - P.W / 128) * BN;
-    bf16* grow_p = P.g + (size_t)grow * P.W + col0;
-    const float* bias = P.bias_cat + it.b_row;
-#pragma unroll 1
-    for (int cc = 0; cc < BN / 32; ++cc) {
-        float v[32];
-        load_acc32(tacc + cc * 32, v);
-        add_bias32(v, bias + cc * 32);
-        store_bf16_32(grow_p + cc * 32, v);
-    }
-}
-
-// a = SiLU(acc + b1)
-__device__ __forceinline__ void epi_g1(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
-    const int col0 = it.nt * BN;
-    bf16* arow = P.a + (size_t)grow * P.W + col0;
-    const float* bias = P.bias_cat + it.b_row;
-#pragma unroll 1
-    for (int cc = 0; cc < BN / 32; ++cc) {
-        float v[32];
-        load_acc32(tacc + cc * 32, v);
-        add_bias32(v, bias + cc * 32);
+            for (int i = 0; i < 32; ++i) st.add(v[i]);
+            float cv[32];
+            slabF_read(bufF, r, cv);
+            slabF_write(bufF, r, v);
+            add_bias32(cv, P.temb + (size_t)it.k * P.W + it.nt * BN + cc * 32);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = silu_f(v[i]);
-        store_bf16_32(arow + cc * 32, v);
-    }
-}
-
-// h += g * (acc + b2) ; LN partial statistics of the new h
-__device__ __forceinline__ void epi_g2(const HeadParams& P, const Item& it, uint32_t tacc, int grow) {
-    const int col0 = it.nt * BN;
-    float* hrow = P.h + (size_t)grow * P.W + col0;
-    const bf16* grow_p = P.g + (size_t)grow * P.W + col0;
-    const float* bias = P.bias_cat + it.b_row;
-    Stats st;
-#pragma unroll 1
-    for (int cc = 0; cc < BN / 32; ++cc) {
-        float v[32], gv[32], hv[32];
-        load_acc32(tacc + cc * 32, v);
-        add_bias32(v, bias + cc * 32);
-        load_bf16_32(grow_p + cc * 32, gv);
-        load_f32_32(hrow + cc * 32, hv);
+            for (int i = 0; i < 32; ++i) cv[i] = silu_f(cv[i]);
+            slabH_write(bufH, r, cv);
+            break;
+        }
+        case OP_MOD:
+        case OP_FMOD: {
+            const float* bias = P.bias_cat + it.b_row;
+            if (it.type == OP_FMOD || it.nt < P.W / 128) {   // u = LN(h) * (1 + scale) + shift
+                float sc[32], hv[32];
+                load_acc32(tacc + cc * 32, v);
+                load_acc32(tacc + 128 + cc * 32, sc);
+                add_bias32(v, bias + cc * 32);
+                add_bias32(sc, bias + 128 + cc * 32);
+                slabF_read(bufF, r, hv);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) hv[i] = fmaf(gv[i], v[i], hv[i]);
-        if (cc == 0) st.init(hv[0]);
+                for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], v[i]);
+                slabH_write(bufH, r, hv);
+            } else {                                          // g = acc + bias
+                load_acc32(tacc + cc * 32, v);
+                add_bias32(v, bias + cc * 32);
+                slabH_write(bufH, r, v);
+            }
+            break;
+        }
+        case OP_G1: {                         // a = SiLU(acc + b1)
+            load_acc32(tacc + cc * 32, v);
+            add_bias32(v, P.bias_cat + it.b_row + cc * 32);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) st.add(hv[i]);
-        store_f32_32(hrow + cc * 32, hv);
+            for (int i = 0; i < 32; ++i) v[i] = silu_f(v[i]);
+            slabH_write(bufH, r, v);
+            break;
+        }
+        default: {                            // OP_G2: h += g * (acc + b2)
+            float gv[32], hv[32];
+            load_acc32(tacc + cc * 32, v);
+            add_bias32(v, P.bias_cat + it.b_row + cc * 32);
+            slabH_read(bufH, r, gv);
+            slabF_read(bufF, r, hv);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) hv[i] = fmaf(gv[i], v[i], hv[i]);
+            if (cc == 0) st.init(hv[0]);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) st.add(hv[i]);
+            slabF_write(bufF, r, hv);
+            break;
+        }
     }
-    P.stats[(size_t)grow * P.NT + it.nt] = st.finish(BN);
 }
 
 // v = acc + bout ; x += dt_k v ; bf16 copy for the next in-projection ; last step: out[idx[j]] = x
@@ -468,13 +481,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = ptx::smem_u32(smem);
-    const uint32_t bars = smem_base + STAGES * STAGE_BYTES;
+    const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;      // 1024-aligned
+    const uint32_t bars = epi_base + EPI_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
     auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
     const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 5));
+    auto epi_bar = [&](int w, int b) { return bars + 8u * (2 * STAGES + 5 + w * EPI_NB + b); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + EPI_BYTES + 8 * NUM_BARS);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -498,6 +513,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             ptx::mbar_init(tempty_bar(b), 4);
         }
         ptx::mbar_init(drain_bar, 1);
+        for (int w = 0; w < 4; ++w)
+            for (int b = 0; b < EPI_NB; ++b) ptx::mbar_init(epi_bar(w, b), 1);
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -595,10 +612,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;  // row of the tile owned by this thread
         const bool leader = (threadIdx.x == 64);
+        const uint32_t my_buf = epi_base + (uint32_t)ewarp * EPI_NB * EPI_BUF;
+        uint32_t ld_parity = 0;               // bit b: parity to wait for on this warp's barrier b
+        uint32_t ld_pending = 0;              // bit b: a load into buffer b is in flight
         uint32_t acc_iter = 0;
         for (long long item = blockIdx.x; item < total; item += gridDim.x) {
             Item it;
             decode_item(P, MT, item, it);
+            bool fail = false;
             if (it.type == OP_GATHER) {
                 bool ok = true;
                 if (leader && it.abs_m >= P.slots)
@@ -606,39 +627,96 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 if (epi_any(!ok)) break;
                 gather_rows(P, it, ewarp, lane, count);
             } else {
+                // producers of this token tile first: the chunk loads below read what they wrote
+                bool ok = true;
+                if (leader) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
+                if (epi_any(!ok)) break;
+                ptx::fence_proxy_async();
+                const EpiIO io = epi_io(P, it);
+                const bool has_loads = (io.ldF >= 0) || (io.ldH >= 0);
+                const int row0 = it.slot_row0 + quarter * 32;
+                auto issue_load = [&](int cc) {
+                    const int b = cc % EPI_NB;
+                    if (lane == 0) {
+                        const uint32_t bar = epi_bar(ewarp, b);
+                        const uint32_t dst = my_buf + (uint32_t)b * EPI_BUF;
+                        ptx::mbar_arrive_expect_tx(bar, (io.ldF >= 0 ? SLAB_F : 0) + (io.ldH >= 0 ? SLAB_H : 0));
+                        if (io.ldF >= 0) ptx::tma_load_2d(dst, P.maps + io.ldF, bar, io.ldF_col + 32 * cc, row0);
+                        if (io.ldH >= 0)
+                            ptx::tma_load_2d(dst + SLAB_F, P.maps + io.ldH, bar, io.ldH_col + 32 * cc, row0);
+                    }
+                    ld_pending |= 1u << b;
+                };
+                if (has_loads) {
+                    issue_load(0);
+                    if (io.nch > 1) issue_load(1);
+                }
                 const uint32_t buf = acc_iter & 1u;
                 const uint32_t acc_phase = (acc_iter >> 1) & 1u;
-                bool ok = wait_mbar(tfull_bar(buf), acc_phase, P);
-                // the operands of this item arrived, so its producers are done; take the acquire
-                // in this thread too before reading what other CTAs wrote
-                if (ok && leader) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
-                if (epi_any(!ok)) break;
+                ok = wait_mbar(tfull_bar(buf), acc_phase, P);
+                ok = __all_sync(0xffffffffu, ok);
+                fail = !ok;
                 ptx::tc_fence_after();
                 const uint32_t tacc = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
                 const int grow = it.slot_row0 + row;
-                switch (it.type) {
-                    case OP_COND: epi_cond(P, it, tacc, grow); break;
-                    case OP_IN: epi_in(P, it, tacc, grow); break;
-                    case OP_MOD:
-                        if (it.nt < P.W / 128) epi_mod_ss(P, it, tacc, grow);
-                        else epi_mod_g(P, it, tacc, grow);
-                        break;
-                    case OP_FMOD: epi_mod_ss(P, it, tacc, grow); break;
-                    case OP_G1: epi_g1(P, it, tacc, grow); break;
-                    case OP_G2: epi_g2(P, it, tacc, grow); break;
-                    default: epi_out(P, it, tacc, grow, it.abs_m * BM + row, count); break;
+                if (it.type == OP_OUT) {
+                    if (!fail) epi_out(P, it, tacc, grow, it.abs_m * BM + row, count);
+                } else {
+                    Stats st;
+                    st.init(0.f);
+                    float mean = 0.f, rstd = 0.f;
+                    if (it.type == OP_FMOD || (it.type == OP_MOD && it.nt < P.W / 128)) row_mean_rstd(P, grow, mean, rstd);
+#pragma unroll 1
+                    for (int cc = 0; cc < io.nch; ++cc) {
+                        const int b = cc % EPI_NB;
+                        const uint32_t bufF = my_buf + (uint32_t)b * EPI_BUF;
+                        const uint32_t bufH = bufF + SLAB_F;
+                        if (has_loads) {
+                            bool okw = wait_mbar(epi_bar(ewarp, b), (ld_parity >> b) & 1u, P);
+                            okw = __all_sync(0xffffffffu, okw);
+                            ld_parity ^= 1u << b;
+                            ld_pending &= ~(1u << b);
+                            fail |= !okw;
+                        } else {
+                            // the store that last used this buffer must have finished reading it
+                            if (lane == 0) ptx::bulk_wait_read<EPI_NB - 1>();
+                            __syncwarp();
+                        }
+                        epi_chunk(P, it, cc, tacc, bufF, bufH, lane, st, mean, rstd);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (has_loads && cc + 2 < io.nch) {
+                            // buffer of chunk cc+2 = buffer of chunk cc-1: its store must be done reading
+                            if (lane == 0) ptx::bulk_wait_read<0>();
+                            issue_load(cc + 2);
+                        }
+                        if (lane == 0) {
+                            if (io.stF >= 0) ptx::tma_store_2d(P.maps + io.stF, bufF, io.stF_col + 32 * cc, row0);
+                            if (io.stH >= 0) ptx::tma_store_2d(P.maps + io.stH, bufH, io.stH_col + 32 * cc, row0);
+                            ptx::bulk_commit();
+                        }
+                    }
+                    if (it.type == OP_IN || it.type == OP_G2) P.stats[(size_t)grow * P.NT + it.nt] = st.finish(BN);
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
                 ++acc_iter;
+                if (lane == 0) ptx::bulk_wait<0>();   // this warp's stores are performed
+                __syncwarp();
             }
             // publish: this item's global writes, then one tick of the token tile's counter
             __threadfence();
             ptx::fence_proxy_async();
-            ptx::named_barrier_sync(1, EPI_THREADS);
+            const bool any_fail = epi_any(fail);
+            if (any_fail) break;
             if (leader) ptx::red_release_gpu_add(P.counters + it.abs_m, 1);
         }
+        // own copies in flight: loads that were issued but never consumed, stores not yet done
+        for (int b = 0; b < EPI_NB; ++b)
+            if (ld_pending & (1u << b)) wait_mbar(epi_bar(ewarp, b), (ld_parity >> b) & 1u, P, kDrainLimitNs);
+        if (lane == 0) ptx::bulk_wait<0>();
+        __syncwarp();
     }
 
     ptx::tc_fence_before();
@@ -753,6 +831,21 @@ bool make_map(CUtensorMap* m, void* base, uint64_t rows, uint64_t cols, uint32_t
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// epilogue slab maps: box = [32 rows][32 columns]; fp32 rows are 128 B (128-byte swizzle), bf16 rows
+// 64 B (64-byte swizzle)
+bool make_slab_map(CUtensorMap* m, void* base, uint64_t rows, uint64_t cols, bool fp32) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const uint64_t esz = fp32 ? 4 : 2;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * esz};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides,
+              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, fp32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline float bf16_bits_to_float(uint16_t b) {
@@ -1000,6 +1093,12 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, BN);
         ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, BN);
         ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C);
+        ok &= make_slab_map(&maps[EMAP_H], H->h, R, W, true);
+        ok &= make_slab_map(&maps[EMAP_C], H->c, R, W, true);
+        ok &= make_slab_map(&maps[EMAP_S], H->s, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_U], H->u, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_A], H->a, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_G], H->g, R, W, false);
         if (!ok) {
             free_all(H);
             delete H;
