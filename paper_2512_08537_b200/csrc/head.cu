@@ -35,10 +35,15 @@ using bf16 = __nv_bfloat16;
 constexpr int BM = 128;           // tokens per tile
 constexpr int BN = 256;           // output columns per tile (UMMA N)
 constexpr int BK = 64;            // K slice per pipeline stage (128 bytes of bf16: one swizzle row)
-constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+// One CTA per tile: 3 stages of (A 16 KB + B 32 KB). CTA pair (tcgen05 cta_group::2, the two CTAs of
+// a cluster work on two token tiles x one column tile): each CTA stages its own A and HALF of B,
+// 4 stages of (16 KB + 16 KB).
+template <bool PAIR> struct Cfg {
+    static constexpr int STAGES = PAIR ? 4 : 3;
+    static constexpr int B_ROWS = PAIR ? BN / 2 : BN;
+    static constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;
+};
 // epilogue staging: every epilogue warp owns EPI_NB buffers, each one fp32 slab (32 rows x 128 B,
 // 128-byte swizzle) plus one bf16 slab (32 rows x 64 B, 64-byte swizzle), filled and drained by TMA
 constexpr int EPI_NB = 3;
@@ -46,8 +51,11 @@ constexpr int SLAB_F = 32 * 128;
 constexpr int SLAB_H = 32 * 64;
 constexpr int EPI_BUF = SLAB_F + SLAB_H;
 constexpr int EPI_BYTES = 4 * EPI_NB * EPI_BUF;
-constexpr int NUM_BARS = 2 * STAGES + 5 + 4 * EPI_NB;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*align slack*/ + 8 * NUM_BARS + 16;
+constexpr int MAX_STAGES = 4;
+constexpr int NUM_BARS = 2 * MAX_STAGES + 5 + 4 * EPI_NB;
+template <bool PAIR> constexpr int smem_bytes() {
+    return Cfg<PAIR>::STAGES * Cfg<PAIR>::STAGE_BYTES + EPI_BYTES + 1024 /*align slack*/ + 8 * NUM_BARS + 16;
+}
 constexpr int NUM_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
 constexpr int XB_COLS = 64;       // x is fed to the in-projection as bf16, K padded to one slice
 constexpr int KMAX = 64;
@@ -73,7 +81,7 @@ struct StepOp {
 };
 
 struct HeadParams {
-    int C, Dc, W, L, K, NT, TG, slots;      // NT = W/256, slots = 2*TG token tiles of scratch
+    int C, Dc, W, L, K, NT, TG, slots;      // NT = W/256, TG token tiles per group (even), slots = 2*TG
     int T_pro, T_step, T_chain, n_step_ops;
     int max_tokens;
     const StepOp* step_ops;
@@ -166,12 +174,17 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-__device__ __forceinline__ void decode_item(const HeadParams& P, int MT, long long item, Item& it) {
-    const long long per_group = (long long)P.TG * P.T_chain;
+// Item `item` of the static list. A unit is one token tile (one CTA per tile) or two consecutive
+// token tiles (CTA pair); MTu = units in this call, upt = token tiles per unit, rank = this CTA's
+// tile within the unit.
+__device__ __forceinline__ void decode_item(const HeadParams& P, int MTu, int upt, int rank, long long item,
+                                            Item& it) {
+    const int TGu = P.TG / upt;
+    const long long per_group = (long long)TGu * P.T_chain;
     const int grp = (int)(item / per_group);
     int r = (int)(item - (long long)grp * per_group);
-    const int m0 = grp * P.TG;
-    const int mtg = min(P.TG, MT - m0);
+    const int m0 = grp * TGu;
+    const int mtg = min(TGu, MTu - m0);
     const int pro = mtg * P.T_pro;
     int m;
     if (r < pro) {
@@ -205,7 +218,7 @@ __device__ __forceinline__ void decode_item(const HeadParams& P, int MT, long lo
         it.b_row = op.b_row0 + it.nt * BN;
         it.kblocks = op.kblocks; it.umma_n = op.umma_n; it.block = op.block;
     }
-    it.abs_m = m0 + m;
+    it.abs_m = (m0 + m) * upt + rank;
     it.slot_row0 = (it.abs_m % P.slots) * BM;
 }
 
@@ -475,24 +488,34 @@ __device__ __forceinline__ void gather_rows(const HeadParams& P, const Item& it,
 }
 
 // ------------------------------------------------------------------------------------------
-// the persistent kernel
+// the persistent kernel. PAIR = false: every CTA works alone (tcgen05 cta_group::1).
+// PAIR = true: clusters of two CTAs; both load their own token tile (A) and half of the weight
+// tile (B); the even CTA issues cta_group::2 MMAs that read both CTAs' shared memory and write
+// 128 accumulator rows into each CTA's TMEM; every CTA runs the epilogue of its own token tile.
 // ------------------------------------------------------------------------------------------
+template <bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_constant__ HeadParams P) {
+    constexpr int STAGES = Cfg<PAIR>::STAGES;
+    constexpr int STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = ptx::smem_u32(smem);
     const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;      // 1024-aligned
     const uint32_t bars = epi_base + EPI_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
-    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
-    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
-    auto epi_bar = [&](int w, int b) { return bars + 8u * (2 * STAGES + 5 + w * EPI_NB + b); };
+    auto empty_bar = [&](int s) { return bars + 8u * (MAX_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * MAX_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * MAX_STAGES + 2 + b); };
+    const uint32_t drain_bar = bars + 8u * (2 * MAX_STAGES + 4);
+    auto epi_bar = [&](int w, int b) { return bars + 8u * (2 * MAX_STAGES + 5 + w * EPI_NB + b); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + EPI_BYTES + 8 * NUM_BARS);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const int rank = PAIR ? (int)ptx::cluster_ctarank() : 0;       // tile of the unit this CTA owns
+    constexpr int UPT = PAIR ? 2 : 1;                              // token tiles per unit
+    const int unit_id = (int)blockIdx.x / UPT;
+    const int n_units = (int)gridDim.x / UPT;
 
     int count = __ldg(P.count);
     if (count > P.max_tokens) {
@@ -501,7 +524,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     }
     if (count < 0) count = 0;
     const int MT = (count + BM - 1) / BM;
-    const long long total = (long long)MT * P.T_chain;
+    const int MTu = (MT + UPT - 1) / UPT;      // an odd last tile gets an all-padding partner
+    const long long total = (long long)MTu * P.T_chain;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -510,7 +534,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 4);
+            ptx::mbar_init(tempty_bar(b), 4 * UPT);   // epilogue warps of every CTA of the unit
         }
         ptx::mbar_init(drain_bar, 1);
         for (int w = 0; w < 4; ++w)
@@ -518,94 +542,131 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
-        ptx::tmem_relinquish();
+        if (PAIR) {
+            ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    bool aborted = false;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         int stage = 0;
         uint32_t phase = 0;
         uint32_t issued = 0, issued_parity = 0;
-        for (long long item = blockIdx.x; item < total; item += gridDim.x) {
+        for (long long item = unit_id; item < total; item += n_units) {
             Item it;
-            decode_item(P, MT, item, it);
+            decode_item(P, MTu, UPT, rank, item, it);
             if (it.type == OP_GATHER) continue;
             bool ok = true;
             if (lane == 0) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            if (!ok) { aborted = true; break; }
             ptx::fence_proxy_async();
             const void* map_a = P.maps + it.map_a;
             const void* map_b = P.maps + it.map_b;
-            const uint32_t tx = A_BYTES + (uint32_t)it.umma_n * BK * 2;
+            const int b_rows = it.umma_n / UPT;                       // rows of B this CTA stages
+            const uint32_t tx = (uint32_t)UPT * (A_BYTES + (uint32_t)b_rows * BK * 2);
             for (int kb = 0; kb < it.kblocks; ++kb) {
                 ok = wait_mbar(empty_bar(stage), phase ^ 1u, P);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (lane == 0) {
                     const uint32_t sa = smem_base + stage * STAGE_BYTES;
-                    ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-                    ptx::tma_load_2d(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
-                    ptx::tma_load_2d(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row);
+                    if (PAIR) {
+                        // the even CTA arms its barrier for the bytes of both CTAs
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                        ptx::tma_load_2d_pair(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
+                        ptx::tma_load_2d_pair(sa + A_BYTES, map_b, full_bar(stage), kb * BK,
+                                              it.b_row + rank * b_rows);
+                    } else {
+                        ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                        ptx::tma_load_2d(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
+                        ptx::tma_load_2d(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row);
+                    }
                 }
                 issued |= 1u << stage;
                 issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
-            if (!ok) break;
+            if (!ok) { aborted = true; break; }
         }
-        // own copies in flight: every stage's last issue must have landed before the CTA exits
-        for (int s = 0; s < STAGES; ++s)
-            if (issued & (1u << s)) wait_mbar(full_bar(s), (issued_parity >> s) & 1u, P, kDrainLimitNs);
+        // own copies in flight must have landed before the CTA exits. Alone (or as the even CTA)
+        // the full barriers are local: wait for every stage's last issue. The odd CTA's loads are
+        // counted on the even CTA's barriers; after a normal run they were all consumed, after an
+        // abort it simply waits out a bounded time that covers any TMA latency.
+        if (!PAIR || rank == 0) {
+            for (int s = 0; s < STAGES; ++s)
+                if (issued & (1u << s)) wait_mbar(full_bar(s), (issued_parity >> s) & 1u, P, kDrainLimitNs);
+        } else if (aborted) {
+            const uint64_t t0 = ptx::globaltimer_ns();
+            while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        int stage = 0;
-        uint32_t phase = 0;
-        uint32_t acc_iter = 0;
-        for (long long item = blockIdx.x; item < total; item += gridDim.x) {
-            Item it;
-            decode_item(P, MT, item, it);
-            if (it.type == OP_GATHER) continue;
-            const uint32_t buf = acc_iter & 1u;
-            const uint32_t acc_phase = (acc_iter >> 1) & 1u;
-            bool ok = wait_mbar(tempty_bar(buf), acc_phase ^ 1u, P);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            const uint32_t d_tmem = tmem_base + buf * BN;
-            const uint32_t idesc = ptx::idesc_bf16_f32(BM, (uint32_t)it.umma_n);
-            for (int kb = 0; kb < it.kblocks; ++kb) {
-                ok = wait_mbar(full_bar(stage), phase, P);
+        // ---------------- MMA issuer (the even CTA of a pair issues for both) ----------------
+        if (!PAIR || rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t acc_iter = 0;
+            for (long long item = unit_id; item < total; item += n_units) {
+                Item it;
+                decode_item(P, MTu, UPT, rank, item, it);
+                if (it.type == OP_GATHER) continue;
+                const uint32_t buf = acc_iter & 1u;
+                const uint32_t acc_phase = (acc_iter >> 1) & 1u;
+                bool ok = wait_mbar(tempty_bar(buf), acc_phase ^ 1u, P);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t sa = smem_base + stage * STAGE_BYTES;
-                    const uint64_t da = ptx::smem_desc_sw128(sa);
-                    const uint64_t db = ptx::smem_desc_sw128(sa + A_BYTES);
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                const uint32_t idesc = ptx::idesc_bf16_f32(BM * UPT, (uint32_t)it.umma_n);
+                for (int kb = 0; kb < it.kblocks; ++kb) {
+                    ok = wait_mbar(full_bar(stage), phase, P);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                        const uint64_t da = ptx::smem_desc_sw128(sa);
+                        const uint64_t db = ptx::smem_desc_sw128(sa + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        ptx::mma_f16_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
-                                        (kb | k) != 0 ? 1u : 0u);
-                    ptx::mma_commit(empty_bar(stage));
+                        for (int k = 0; k < BK / 16; ++k) {
+                            if (PAIR)
+                                ptx::mma_f16_ss_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
+                                                     (kb | k) != 0 ? 1u : 0u);
+                            else
+                                ptx::mma_f16_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
+                                                (kb | k) != 0 ? 1u : 0u);
+                        }
+                        if (PAIR) ptx::mma_commit_pair_mc(empty_bar(stage), 3);   // frees the stage in both CTAs
+                        else ptx::mma_commit(empty_bar(stage));
+                    }
+                    __syncwarp();
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (lane == 0) {
+                    if (PAIR) ptx::mma_commit_pair_mc(tfull_bar(buf), 3);
+                    else ptx::mma_commit(tfull_bar(buf));
                 }
                 __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                ++acc_iter;
             }
-            if (!ok) break;
-            if (lane == 0) ptx::mma_commit(tfull_bar(buf));
+            // all MMAs this thread issued must be done before TMEM is freed
+            if (lane == 0) {
+                if (PAIR) ptx::mma_commit_pair(drain_bar);
+                else ptx::mma_commit(drain_bar);
+            }
             __syncwarp();
-            ++acc_iter;
+            wait_mbar(drain_bar, 0, P, kDrainLimitNs);
         }
-        // all MMAs this thread issued must be done before TMEM is freed
-        if (lane == 0) ptx::mma_commit(drain_bar);
-        __syncwarp();
-        wait_mbar(drain_bar, 0, P, kDrainLimitNs);
     } else {
         // ---------------- epilogue warps ----------------
         const int ewarp = warp - 2;           // 0..3
@@ -616,9 +677,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         uint32_t ld_parity = 0;               // bit b: parity to wait for on this warp's barrier b
         uint32_t ld_pending = 0;              // bit b: a load into buffer b is in flight
         uint32_t acc_iter = 0;
-        for (long long item = blockIdx.x; item < total; item += gridDim.x) {
+        for (long long item = unit_id; item < total; item += n_units) {
             Item it;
-            decode_item(P, MT, item, it);
+            decode_item(P, MTu, UPT, rank, item, it);
             bool fail = false;
             if (it.type == OP_GATHER) {
                 bool ok = true;
@@ -700,7 +761,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
+                if (lane == 0) {
+                    if (PAIR) ptx::mbar_arrive_even_cta(tempty_bar(buf));
+                    else ptx::mbar_arrive(tempty_bar(buf));
+                }
                 ++acc_iter;
                 if (lane == 0) ptx::bulk_wait<0>();   // this warp's stores are performed
                 __syncwarp();
@@ -720,10 +784,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     }
 
     ptx::tc_fence_before();
-    __syncthreads();
+    // nobody leaves while its partner may still signal its barriers or read its shared memory
+    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, 512);
+        if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512);
+        else ptx::tmem_dealloc(tmem_base, 512);
     }
 }
 
@@ -859,7 +925,7 @@ inline float bf16_bits_to_float(uint16_t b) {
 
 struct ardiff_head {
     ardiff_head_desc d;
-    int device, n_sm, grid;
+    int device, n_sm, grid, pair;
     int NT, TG, slots, T_pro, T_step, T_chain, n_step_ops;
     int64_t max_tiles;
     std::vector<void*> allocs;
@@ -958,26 +1024,51 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     H->max_tiles = (d.max_tokens + BM - 1) / BM;
     if (H->max_tiles < 1) H->max_tiles = 1;
 
-    // grid: one CTA per SM, all co-resident (cooperative launch)
-    if (cudaFuncSetAttribute(head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
-        delete H;
-        return ARDIFF_ERR_CUDA;
-    }
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, head_kernel, NUM_THREADS, SMEM_BYTES) != cudaSuccess ||
-        per_sm < 1) {
-        delete H;
-        return ARDIFF_ERR_CUDA;
+    // grid: one CTA per SM, all co-resident (cooperative launch). Default: CTA pairs (clusters of 2).
+    H->pair = env_int("ARDIFF_HEAD_PAIR", 1) != 0;
+    {
+        bool ok = cudaFuncSetAttribute(head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       smem_bytes<false>()) == cudaSuccess;
+        ok &= cudaFuncSetAttribute(head_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   smem_bytes<true>()) == cudaSuccess;
+        int per_sm = 0;
+        ok = ok && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, head_kernel<false>, NUM_THREADS,
+                                                                 smem_bytes<false>()) == cudaSuccess && per_sm >= 1;
+        if (!ok) {
+            (void)cudaGetLastError();
+            delete H;
+            return ARDIFF_ERR_CUDA;
+        }
     }
     H->grid = env_int("ARDIFF_HEAD_GRID", H->n_sm);
     if (H->grid < 1 || H->grid > H->n_sm) H->grid = H->n_sm;
+    if (H->pair) {
+        // every cluster of two must be resident at once
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3(H->grid & ~1); cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = smem_bytes<true>(); cfg.attrs = at; cfg.numAttrs = 1;
+        int max_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, head_kernel<true>, &cfg) != cudaSuccess || max_clusters < 1) {
+            (void)cudaGetLastError();
+            H->pair = 0;
+        } else {
+            H->grid &= ~1;
+            if (H->grid > 2 * max_clusters) H->grid = 2 * max_clusters;
+        }
+    }
+    const int units = H->pair ? H->grid / 2 : H->grid;
 
-    // token tiles per group: enough column tiles per layer to keep every CTA busy while the
+    // token tiles per group: enough column tiles per layer to keep every unit busy while the
     // layer before it drains (about 1.5 grids of items), capped by what exists
-    int tg = (3 * H->grid / 2 + H->NT - 1) / H->NT;
+    int tg = ((3 * units / 2 + H->NT - 1) / H->NT) * (H->pair ? 2 : 1);
     tg = env_int("ARDIFF_HEAD_TG", tg);
     if (tg < 1) tg = 1;
     if ((int64_t)tg > H->max_tiles) tg = (int)H->max_tiles;
+    if (H->pair) tg = (tg + 1) & ~1;
     H->TG = tg;
     H->slots = 2 * tg;
     const size_t R = (size_t)H->slots * BM;
@@ -1049,7 +1140,7 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     TRY(dev_alloc(H, &H->c, R * W, true));
     TRY(dev_alloc(H, &H->h, R * W, true));
     TRY(dev_alloc(H, &H->stats, R * H->NT, true));
-    TRY(dev_alloc(H, &H->counters, (size_t)H->max_tiles, true));
+    TRY(dev_alloc(H, &H->counters, (size_t)H->max_tiles + 2, true));
     TRY(dev_alloc(H, &H->status, 2, true));
 
     // ---- op table of one step ----
@@ -1089,10 +1180,11 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         ok &= make_map(&maps[MAP_S], H->s, R, W, BM);
         ok &= make_map(&maps[MAP_U], H->u, R, W, BM);
         ok &= make_map(&maps[MAP_A], H->a, R, W, BM);
-        ok &= make_map(&maps[MAP_WC], H->Wc, W, Dc, BN);
-        ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, BN);
-        ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, BN);
-        ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C);
+        const uint32_t bdiv = H->pair ? 2 : 1;   // a CTA of a pair stages half of the weight tile's rows
+        ok &= make_map(&maps[MAP_WC], H->Wc, W, Dc, BN / bdiv);
+        ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, BN / bdiv);
+        ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, BN / bdiv);
+        ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C / bdiv);
         ok &= make_slab_map(&maps[EMAP_H], H->h, R, W, true);
         ok &= make_slab_map(&maps[EMAP_C], H->c, R, W, true);
         ok &= make_slab_map(&maps[EMAP_S], H->s, R, W, false);
@@ -1154,7 +1246,7 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
                                                                                   H->temb_hidden);
     temb_out_kernel<<<dim3((W + 7) / 8, K), 256, 0, st>>>(H->Wt2, H->bt2, W, H->temb_hidden, H->temb);
     launches += 2;
-    if (cudaMemsetAsync(H->counters, 0, sizeof(int) * (size_t)H->max_tiles, st) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    if (cudaMemsetAsync(H->counters, 0, sizeof(int) * ((size_t)H->max_tiles + 2), st) != cudaSuccess) return ARDIFF_ERR_CUDA;
     if (cudaMemsetAsync(H->status + 1, 0, sizeof(int), st) != cudaSuccess) return ARDIFF_ERR_CUDA;
 
     HeadParams P;
@@ -1170,13 +1262,30 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
     P.counters = H->counters; P.status = H->status; P.abort_flag = H->status + 1;
     for (int k = 0; k < K; ++k) P.dt[k] = (float)((double)t_sched[k + 1] - (double)t_sched[k]);
 
-    void* args[] = {&P};
     ardiff_head* Hm = const_cast<ardiff_head*>(H);
     if (H->timing) cudaEventRecord(H->ev0, st);
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(head_kernel), dim3(H->grid), dim3(NUM_THREADS), args,
-                                    SMEM_BYTES, st) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return ARDIFF_ERR_CUDA;
+    {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cudaLaunchAttribute at[2];
+        int na = 0;
+        at[na].id = cudaLaunchAttributeCooperative;
+        at[na].val.cooperative = 1;
+        ++na;
+        if (H->pair) {
+            at[na].id = cudaLaunchAttributeClusterDimension;
+            at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+            ++na;
+        }
+        cfg.gridDim = dim3(H->grid); cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = H->pair ? smem_bytes<true>() : smem_bytes<false>();
+        cfg.stream = st; cfg.attrs = at; cfg.numAttrs = na;
+        cudaError_t e = H->pair ? cudaLaunchKernelEx(&cfg, head_kernel<true>, P)
+                                : cudaLaunchKernelEx(&cfg, head_kernel<false>, P);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return ARDIFF_ERR_CUDA;
+        }
     }
     if (H->timing) {
         cudaEventRecord(H->ev1, st);
