@@ -925,7 +925,7 @@ inline float bf16_bits_to_float(uint16_t b) {
 
 struct ardiff_head {
     ardiff_head_desc d;
-    int device, n_sm, grid, pair;
+    int device, n_sm, grid, pair, coop;
     int NT, TG, slots, T_pro, T_step, T_chain, n_step_ops;
     int64_t max_tiles;
     std::vector<void*> allocs;
@@ -1026,6 +1026,10 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
 
     // grid: one CTA per SM, all co-resident (cooperative launch). Default: CTA pairs (clusters of 2).
     H->pair = env_int("ARDIFF_HEAD_PAIR", 1) != 0;
+    // The cooperative attribute makes the launch fail instead of start when the grid cannot be
+    // co-resident. ARDIFF_HEAD_COOP=0 drops it for tools that cannot replay such launches (the
+    // grid is still sized to be co-resident on an otherwise idle device, and every wait is bounded).
+    H->coop = env_int("ARDIFF_HEAD_COOP", 1) != 0;
     {
         bool ok = cudaFuncSetAttribute(head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        smem_bytes<false>()) == cudaSuccess;
@@ -1269,9 +1273,11 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
         memset(&cfg, 0, sizeof(cfg));
         cudaLaunchAttribute at[2];
         int na = 0;
-        at[na].id = cudaLaunchAttributeCooperative;
-        at[na].val.cooperative = 1;
-        ++na;
+        if (H->coop) {
+            at[na].id = cudaLaunchAttributeCooperative;
+            at[na].val.cooperative = 1;
+            ++na;
+        }
         if (H->pair) {
             at[na].id = cudaLaunchAttributeClusterDimension;
             at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
