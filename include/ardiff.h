@@ -68,6 +68,34 @@ int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, float tau, ui
                            int32_t* idx, int32_t* count, float* entropy, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Entropy gate for callers that cannot allocate device memory. (The paper has no counterpart:
+ * this is a packaging variant of ardiff_entropy_gate, same operation, same results.)
+ *
+ * Who needs it: a process whose own pool owns all device memory and forbids a library to
+ * call cudaMalloc behind its back; a caller between cudaStreamBeginCapture and EndCapture,
+ * where allocating is an error; a latency-critical loop that must not meet the allocator's
+ * lock or the device-wide synchronisation an allocation may imply. ardiff_entropy_gate
+ * allocates its per-block count array on its first call on a device; this entry point never
+ * calls cudaMalloc, cudaFree or any allocating routine. Its scratch is a fixed array of
+ * ARDIFF_GATE_NOALLOC_MAX_BLOCKS int32 (4 KB) compiled into the library as a __device__
+ * variable, so every GPU that loads the library holds it until the process exits.
+ *
+ * Arguments, layouts, alignment rules and error codes are those of ardiff_entropy_gate, with
+ * one more limit: n <= ARDIFF_GATE_NOALLOC_MAX_TOKENS, else ARDIFF_ERR_SHAPE and nothing is
+ * launched (the fixed number of blocks would otherwise each walk an ever longer token range).
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress,
+ * with that device current); make that first call before any stream capture starts.
+ * All calls on one device share the one array. Every call overwrites the entries it uses
+ * before it reads them, so nothing needs clearing between calls and back-to-back calls on one
+ * stream are safe; two calls that can run on the GPU at the same time (different streams
+ * with no event between them, or mixed host threads) race on it and give undefined idx/count.
+ * ------------------------------------------------------------------------------------- */
+#define ARDIFF_GATE_NOALLOC_MAX_BLOCKS 1024
+#define ARDIFF_GATE_NOALLOC_MAX_TOKENS (1 << 24)
+int ardiff_entropy_gate_noalloc(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask,
+                                int32_t* idx, int32_t* count, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * Diffusion / flow head.
  *
  * Operation (the head call "x = Diff_theta(x_t | t, z)" of the AR+Diffusion hybrid

@@ -130,6 +130,32 @@ def ardiff_entropy_gate(feat, tau: float, mask=None, idx=None, count=None, entro
     return mask, idx, count, entropy
 
 
+GATE_NOALLOC_MAX_BLOCKS = 1024
+GATE_NOALLOC_MAX_TOKENS = 1 << 24
+
+
+def ardiff_entropy_gate_noalloc(feat, tau: float, mask, idx, count, stream=None):
+    """The gate for callers that may not allocate device memory (a process whose own pool owns the
+    device, code inside a stream capture, a latency-critical loop): same kernels and results as
+    ardiff_entropy_gate, but the library's scratch is a fixed __device__ array instead of a
+    cudaMalloc on first use. Because nothing may be allocated, the caller passes every output
+    (mask u8 [n], idx i32 [n], count i32 [1]); there is no entropy output. n is limited to
+    GATE_NOALLOC_MAX_TOKENS. Calls on one device share the scratch: do not let two overlap."""
+    import torch
+    assert feat.is_cuda and feat.dtype == torch.bfloat16 and feat.dim() == 2 and feat.is_contiguous()
+    fn = lib().ardiff_entropy_gate_noalloc
+    if fn.argtypes is None:
+        vp = ctypes.c_void_p
+        fn.restype = ctypes.c_int
+        fn.argtypes = [vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, vp, vp, vp, vp]
+    n, d = feat.shape
+    with torch.cuda.device(feat.device):
+        rc = fn(feat.data_ptr(), n, d, float(tau), mask.data_ptr(), idx.data_ptr(), count.data_ptr(),
+                _stream_ptr(stream))
+    _check(rc, "ardiff_entropy_gate_noalloc")
+    return mask, idx, count
+
+
 class Head:
     """Owns an ardiff_head handle (device weights + scratch)."""
 
