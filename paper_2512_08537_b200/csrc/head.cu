@@ -1,19 +1,23 @@
-// K-step AdaLN residual-MLP flow head for sm_100a: one persistent cooperative kernel.
+// K-step AdaLN residual-MLP flow head for sm_100a: one persistent kernel of CTA pairs.
 //
 // What it computes (per surviving token; see include/ardiff.h for the formulas): the head call
 // x = Diff_theta(x_t | t, z) of the AR+Diffusion hybrid, conditioned on the token's AR hidden
 // state z and on t, sampled with K Euler flow steps from caller-supplied noise.
 //
-// How: every matrix product of the head is cut into tiles of 128 tokens x 256 output columns.
-// Each tile is one "item": TMA streams the bf16 A (activations) and B (weights) K-slices into a
-// 4-stage shared-memory ring, one thread issues tcgen05.mma (bf16 x bf16 -> fp32) into one of
-// two 256-column TMEM accumulators, and four epilogue warps read the accumulator back with
-// tcgen05.ld and apply the fused tail of that layer (bias, SiLU, LayerNorm+modulation, gated
-// residual, LayerNorm statistics, Euler update, scatter) while the next item's MMAs already run.
-// All items of all layers and steps form one static list ordered so that the activations of a
-// group of token tiles stay in L2; CTA c takes items c, c+grid, ... . A tile of layer l needs all
-// column tiles of layer l-1 of the same 128 tokens: that is tracked with one progress counter per
-// token tile (release/acquire at gpu scope, bounded spins).
+// How: every matrix product of the head is cut into items of 128 tokens x 256 output columns. The two
+// CTAs of a cluster form a unit: each owns one token tile, stages its own A tile (activations) and
+// half of the B tile (weights) per 64-wide K slice by TMA into a 4-stage shared-memory ring, and the
+// even CTA issues tcgen05.mma.cta_group::2 (256 x 256 x 16, bf16 -> fp32) into one of two TMEM
+// accumulators. Eight epilogue warps per CTA read the accumulator back with tcgen05.ld and apply the
+// fused tail of the layer (bias, SiLU, LayerNorm statistics, LayerNorm + modulation, gated residual,
+// Euler update, scatter) while the next item's MMAs run; their global operands and results move as
+// swizzled 32 x 32 slabs by TMA.
+// All items of a call form one static list (a per-step "program" of phases, repeated for every step
+// and every group of token tiles); unit u takes items u, u + units, ... . The modulation GEMM of a
+// block is split: its gate third does not depend on the residual stream, so gate items of block b+1
+// are placed between the dependent phases of block b, where they cover the latency of the chain.
+// Dependencies between items are tracked per token tile by three counters (chain, gates of even
+// blocks, gates of odd blocks) with release/acquire at gpu scope; every wait is bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -32,78 +36,98 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-constexpr int BM = 128;           // tokens per tile
-constexpr int BN = 256;           // output columns per tile (UMMA N)
+constexpr int BM = 128;           // tokens per tile (one CTA)
+constexpr int BN = 256;           // output columns per item (UMMA N)
 constexpr int BK = 64;            // K slice per pipeline stage (128 bytes of bf16: one swizzle row)
 constexpr int A_BYTES = BM * BK * 2;
-// One CTA per tile: 3 stages of (A 16 KB + B 32 KB). CTA pair (tcgen05 cta_group::2, the two CTAs of
-// a cluster work on two token tiles x one column tile): each CTA stages its own A and HALF of B,
-// 4 stages of (16 KB + 16 KB).
-template <bool PAIR> struct Cfg {
-    static constexpr int STAGES = PAIR ? 4 : 3;
-    static constexpr int B_ROWS = PAIR ? BN / 2 : BN;
-    static constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;
-};
+constexpr int B_ROWS = BN / 2;    // rows of the weight tile that one CTA of the pair stages
+constexpr int STAGES = 4;
+constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;   // 32 KB
 // epilogue staging: every epilogue warp owns EPI_NB buffers, each one fp32 slab (32 rows x 128 B,
 // 128-byte swizzle) plus one bf16 slab (32 rows x 64 B, 64-byte swizzle), filled and drained by TMA
-constexpr int EPI_NB = 3;
+constexpr int EPI_WARPS = 8;
+constexpr int EPI_NB = 2;
 constexpr int SLAB_F = 32 * 128;
 constexpr int SLAB_H = 32 * 64;
 constexpr int EPI_BUF = SLAB_F + SLAB_H;
-constexpr int EPI_BYTES = 4 * EPI_NB * EPI_BUF;
-constexpr int MAX_STAGES = 4;
-constexpr int NUM_BARS = 2 * MAX_STAGES + 5 + 4 * EPI_NB;
-template <bool PAIR> constexpr int smem_bytes() {
-    return Cfg<PAIR>::STAGES * Cfg<PAIR>::STAGE_BYTES + EPI_BYTES + 1024 /*align slack*/ + 8 * NUM_BARS + 16;
-}
-constexpr int NUM_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int EPI_BYTES = EPI_WARPS * EPI_NB * EPI_BUF;
+constexpr int DEP_BARS = 8;       // the producer runs at most 6 items ahead of the epilogue
+constexpr int NUM_BARS = 2 * STAGES + 5 + DEP_BARS + EPI_WARPS * EPI_NB;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*align slack*/ + 8 * NUM_BARS + 16;
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
 constexpr int XB_COLS = 64;       // x is fed to the in-projection as bf16, K padded to one slice
 constexpr int KMAX = 64;
+constexpr int CTRS = 4;           // counters per token tile: chain, gates of even blocks, gates of odd blocks, pad
 constexpr uint64_t kWaitLimitNs = 4000000000ull;   // a bounded wait gives up after 4 s
 constexpr uint64_t kDrainLimitNs = 200000000ull;   // waits for own copies in flight at exit
 
-enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_MOD, OP_G1, OP_G2, OP_FMOD, OP_OUT };
+// Optional per-item time stamps of CTA 0 (compile with -DARDIFF_HEAD_PROFILE):
+// trace[(local item number * 3 + role) * 4 + slot] = clock64(); slot 3 = type * 1000 + column tile.
+#ifdef ARDIFF_HEAD_PROFILE
+constexpr int TRACE_ITEMS = 4096;
+#define TRACE(role, slot) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + (slot)] = clock64(); } while (0)
+#define TRACE_TYPE(role) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + 3] = it.type * 1000 + it.nt; } while (0)
+#define TRACE_DECL int trace_n = 0;
+#define TRACE_NEXT() ++trace_n
+#else
+#define TRACE(role, slot)
+#define TRACE_TYPE(role)
+#define TRACE_DECL
+#define TRACE_NEXT()
+#endif
+
+enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_SS, OP_GATE, OP_G1, OP_G2, OP_FSS, OP_OUT, OP_END = 15 };
 enum MapId : int {
     MAP_Z = 0, MAP_XB, MAP_S, MAP_U, MAP_A, MAP_WC, MAP_WIN, MAP_WCAT, MAP_WOUT,   // GEMM operands
-    EMAP_H, EMAP_C, EMAP_S, EMAP_U, EMAP_A, EMAP_G,                                 // epilogue slabs
+    EMAP_H, EMAP_C, EMAP_S, EMAP_U, EMAP_A, EMAP_G0, EMAP_G1,                       // epilogue slabs
     MAP_COUNT
 };
 
-struct StepOp {
+// One phase of the per-step program: `ntiles` column tiles (tile0 ..) of one layer for every token
+// tile of the group.
+struct Phase {
     int type;      // OpType
-    int ntiles;    // column tiles of this op per token tile
-    int cum;       // column tiles of the ops before it within one step
-    int map_a, map_b;
-    int b_row0;    // first row of this op's weights in the B matrix
-    int kblocks;   // K / 64
-    int umma_n;    // 256, or C for the out-projection
     int block;     // residual block index (or -1)
+    int tile0;     // first column tile of the layer this phase covers
+    int ntiles;    // column tiles in this phase
+    int cum;       // column tiles per token tile in the phases before it within one step
+    int b_row0;    // first row of the layer's weights in the B matrix
+    int offA;      // chain items of this step that must be complete (per token tile)
+    int gsel;      // 0: none; 1/2: gate counter (even/odd blocks) bumped (OP_GATE) or awaited (OP_G2)
+    int goff;      // OP_G2: gate items of that parity that must be complete within this step
 };
 
 struct HeadParams {
-    int C, Dc, W, L, K, NT, TG, slots;      // NT = W/256, TG token tiles per group (even), slots = 2*TG
-    int T_pro, T_step, T_chain, n_step_ops;
+    int C, Dc, W, L, K, NT, TGu, slots;     // NT = W/256, TGu = largest group in units, slots = scratch tiles
+    int T_pro, T_step, T_chain;             // items per unit: prologue, one step, whole call
+    int C_pro, C_step, C_total;             // chain-counter items per token tile: prologue, one step, whole call
+    int gcnt[2];                            // gate items per step and token tile with even / odd block index
     int max_tokens;
-    const StepOp* step_ops;
+    const Phase* phases;
+    const uint16_t* cum2phase;              // [T_step]: phase that holds the c-th column tile of a step
     const CUtensorMap* maps;
     const bf16* cond;
     const float* noise;
     const int* idx;
     const int* count;
     float* out;
-    bf16 *z, *xb, *s, *u, *a, *g;
+    bf16 *z, *xb, *s, *u, *a, *g0, *g1;
     float *x, *c, *h;
     float2* stats;
     const float *bias_cat, *bc, *bin, *temb;
     int* counters;
     int* status;
     int* abort_flag;
+    long long* trace;
     float dt[KMAX];
 };
 
+struct Packed { uint32_t w0, w1, w2, w3, w4; };
+
 struct Item {
-    int type, abs_m, slot_row0, nt, k, prior;
-    int map_a, map_b, b_row, kblocks, umma_n, block;
+    int type, abs_m, slot_row0, nt, k, block, gsel;
+    int needA, needB;
+    int map_a, map_b, b_row, kblocks, umma_n;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -133,14 +157,15 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const H
     }
 }
 
-// bounded wait until *ctr >= need (acquire); one thread calls it
-__device__ __forceinline__ bool wait_counter(const int* ctr, int need, const HeadParams& P) {
-    if (ptx::ld_acquire_gpu(ctr) >= need) return true;
+// bounded wait until *c1 >= n1 and (c2 == nullptr or *c2 >= n2) (acquire); one thread calls it
+__device__ __forceinline__ bool wait_counters(const int* c1, int n1, const int* c2, int n2, const HeadParams& P) {
     uint64_t t0 = 0;
-    for (uint32_t it = 1;; ++it) {
-        if (ptx::ld_acquire_gpu(ctr) >= need) return true;
+    for (uint32_t it = 0;; ++it) {
+        const int v1 = ptx::ld_acquire_gpu(c1);
+        const int v2 = c2 ? ptx::ld_acquire_gpu(c2) : n2;
+        if (v1 >= n1 && v2 >= n2) return true;
         if (it > 8) __nanosleep(64);
-        if ((it & 63u) == 0) {
+        if ((it & 63u) == 63u) {
             if (ptx::ld_relaxed_gpu(P.abort_flag) != 0) return false;
             const uint64_t now = ptx::globaltimer_ns();
             if (t0 == 0) t0 = now;
@@ -152,19 +177,6 @@ __device__ __forceinline__ bool wait_counter(const int* ctr, int need, const Hea
     }
 }
 
-__device__ __forceinline__ bool epi_any(bool pred) {  // OR over the 128 epilogue threads
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 2, 128, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r)
-        : "r"((uint32_t)pred)
-        : "memory");
-    return r != 0;
-}
-
 __device__ __forceinline__ float silu_f(float a) { return __fdividef(a, 1.0f + __expf(-a)); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -174,60 +186,103 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// Item `item` of the static list. A unit is one token tile (one CTA per tile) or two consecutive
-// token tiles (CTA pair); MTu = units in this call, upt = token tiles per unit, rank = this CTA's
-// tile within the unit.
-__device__ __forceinline__ void decode_item(const HeadParams& P, int MTu, int upt, int rank, long long item,
-                                            Item& it) {
-    const int TGu = P.TG / upt;
-    const long long per_group = (long long)TGu * P.T_chain;
+// Item `item` of the static list, for the CTA of rank `rank` within its unit. MTu = units (pairs of
+// token tiles) of this call, tgu = units per group (balanced over the groups).
+__device__ __forceinline__ Packed decode_packed(const HeadParams& P, int MTu, int tgu, int rank, long long item,
+                                                long long total) {
+    Packed pk{(uint32_t)OP_END << 24, 0u, 0u, 0u, 0u};
+    if (item >= total) return pk;
+    const long long per_group = (long long)tgu * P.T_chain;
     const int grp = (int)(item / per_group);
     int r = (int)(item - (long long)grp * per_group);
-    const int m0 = grp * TGu;
-    const int mtg = min(TGu, MTu - m0);
+    const int m0 = grp * tgu;
+    const int mtg = min(tgu, MTu - m0);
     const int pro = mtg * P.T_pro;
-    int m;
+    int m, type, nt = 0, k = 0, block = 0, gsel = 0;
+    int needA = 0, needB = 0, b_row = 0;
     if (r < pro) {
-        it.k = 0;
-        it.block = -1;
         if (r < mtg) {
-            it.type = OP_GATHER; m = r; it.nt = 0; it.prior = 0;
-            it.map_a = it.map_b = 0; it.b_row = 0; it.kblocks = 0; it.umma_n = 0;
+            type = OP_GATHER; m = r;
         } else {
             r -= mtg;
             m = r / P.NT;
-            it.nt = r - m * P.NT;
-            it.type = OP_COND; it.prior = 1;
-            it.map_a = MAP_Z; it.map_b = MAP_WC; it.b_row = it.nt * BN;
-            it.kblocks = P.Dc / BK; it.umma_n = BN;
+            nt = r - m * P.NT;
+            type = OP_COND;
+            needA = EPI_WARPS;            // the gather of this token tile
+            b_row = nt * BN;
         }
     } else {
         r -= pro;
         const int per_step = mtg * P.T_step;
-        it.k = r / per_step;
-        r -= it.k * per_step;
-        int o = 0;
-        while (o + 1 < P.n_step_ops && __ldg(&P.step_ops[o + 1].cum) * mtg <= r) ++o;
-        const StepOp op = P.step_ops[o];
-        const int q = r - op.cum * mtg;
-        m = q / op.ntiles;
-        it.nt = q - m * op.ntiles;
-        it.type = op.type;
-        it.prior = P.T_pro + it.k * P.T_step + op.cum;
-        it.map_a = op.map_a; it.map_b = op.map_b;
-        it.b_row = op.b_row0 + it.nt * BN;
-        it.kblocks = op.kblocks; it.umma_n = op.umma_n; it.block = op.block;
+        k = r / per_step;
+        r -= k * per_step;
+        const int c = r / mtg;
+        const Phase p = P.phases[__ldg(P.cum2phase + c)];
+        const int q = r - p.cum * mtg;
+        m = q / p.ntiles;
+        nt = p.tile0 + (q - m * p.ntiles);
+        type = p.type; block = p.block; gsel = p.gsel;
+        needA = EPI_WARPS * (P.C_pro + k * P.C_step + p.offA);
+        if (type == OP_G2) needB = EPI_WARPS * (k * P.gcnt[gsel - 1] + p.goff);
+        b_row = p.b_row0 + nt * BN;
     }
-    it.abs_m = (m0 + m) * upt + rank;
-    it.slot_row0 = (it.abs_m % P.slots) * BM;
+    const int abs_m = (m0 + m) * 2 + rank;
+    pk.w0 = (uint32_t)abs_m | ((uint32_t)type << 24);
+    pk.w1 = (uint32_t)nt | ((uint32_t)k << 8) | ((uint32_t)(block & 0xff) << 16) | ((uint32_t)gsel << 24);
+    pk.w2 = (uint32_t)needA; pk.w3 = (uint32_t)needB; pk.w4 = (uint32_t)b_row;
+    return pk;
 }
 
+__device__ __forceinline__ void unpack_item(const HeadParams& P, const Packed& pk, Item& it) {
+    it.type = (int)(pk.w0 >> 24);
+    it.abs_m = (int)(pk.w0 & 0xffffffu);
+    it.slot_row0 = (it.abs_m % P.slots) * BM;
+    it.nt = (int)(pk.w1 & 0xffu);
+    it.k = (int)((pk.w1 >> 8) & 0xffu);
+    it.block = (int)((pk.w1 >> 16) & 0xffu);
+    it.gsel = (int)(pk.w1 >> 24);
+    it.needA = (int)pk.w2; it.needB = (int)pk.w3; it.b_row = (int)pk.w4;
+    it.kblocks = P.W / BK; it.umma_n = BN; it.map_b = MAP_WCAT; it.map_a = MAP_S;
+    switch (it.type) {
+        case OP_COND: it.map_a = MAP_Z; it.map_b = MAP_WC; it.kblocks = P.Dc / BK; break;
+        case OP_IN: it.map_a = MAP_XB; it.map_b = MAP_WIN; it.kblocks = 1; break;
+        case OP_G1: it.map_a = MAP_U; break;
+        case OP_G2: it.map_a = MAP_A; break;
+        case OP_OUT: it.map_a = MAP_U; it.map_b = MAP_WOUT; it.umma_n = P.C; break;
+        default: break;
+    }
+}
+
+// The items of one CTA, decoded 32 at a time (lane l decodes the l-th of the next 32) and handed
+// out by shuffle. Every lane of the warp calls next() together.
+struct ItemStream {
+    Packed mine;
+    int n = 0;
+    __device__ __forceinline__ bool next(const HeadParams& P, int MTu, int tgu, int rank, int unit_id, int n_units,
+                                         long long total, int lane, Item& it) {
+        if ((n & 31) == 0)
+            mine = decode_packed(P, MTu, tgu, rank, (long long)unit_id + (long long)(n + lane) * n_units, total);
+        Packed cur;
+        const int src = n & 31;
+        cur.w0 = __shfl_sync(0xffffffffu, mine.w0, src);
+        cur.w1 = __shfl_sync(0xffffffffu, mine.w1, src);
+        cur.w2 = __shfl_sync(0xffffffffu, mine.w2, src);
+        cur.w3 = __shfl_sync(0xffffffffu, mine.w3, src);
+        cur.w4 = __shfl_sync(0xffffffffu, mine.w4, src);
+        ++n;
+        if ((cur.w0 >> 24) == (uint32_t)OP_END) return false;
+        unpack_item(P, cur, it);
+        return true;
+    }
+};
+
 // ------------------------------------------------------------------------------------------
-// epilogues. Lane r of an epilogue warp owns row r of the warp's 32-row quarter of the tile (TMEM
-// lane quarter*32 + r). Work goes in chunks of 32 accumulator columns: the chunk's global inputs
-// (h, c: fp32 slab; g: bf16 slab) arrive by TMA in a swizzled shared-memory buffer, the lane reads
-// its own row, combines it with the accumulator chunk, writes the results back into the buffer
-// (in place) and lane 0 hands the buffer to a TMA store. Loads run two chunks ahead.
+// epilogues. Two epilogue warps share each 32-row quarter of the tile (TMEM lane quarter*32 + lane);
+// warp half h of the pair takes accumulator columns [128 h, 128 h + 128). Work goes in chunks of 32
+// accumulator columns: the chunk's global inputs (h, c: fp32 slab; g: bf16 slab) arrive by TMA in a
+// swizzled shared-memory buffer, the lane reads its own row, combines it with the accumulator chunk,
+// writes the results back into the buffer (in place) and lane 0 hands the buffer to a TMA store.
+// Loads run one chunk ahead.
 // ------------------------------------------------------------------------------------------
 struct Stats {
     float p, sd, sq;
@@ -241,38 +296,26 @@ struct Stats {
     }
 };
 
-struct EpiIO {            // what one item's epilogue moves per 32-column chunk (-1: nothing)
-    int nch;              // chunks
-    int ldF, ldF_col;     // fp32 slab load: map id, first column
-    int ldH, ldH_col;     // bf16 slab load
-    int stF, stF_col;     // fp32 slab store
-    int stH, stH_col;     // bf16 slab store
+struct EpiIO {            // what one warp moves per 32-column chunk of one item (-1: nothing)
+    int nch;              // chunks of this warp
+    int acc0;             // accumulator column of the warp's first chunk
+    int col0;             // global column of the warp's first chunk (slabs, biases)
+    int ldF, ldH, stF, stH;   // map ids
 };
 
-__device__ __forceinline__ EpiIO epi_io(const HeadParams& P, const Item& it) {
-    EpiIO io{BN / 32, -1, 0, -1, 0, -1, 0, -1, 0};
-    const int col0 = it.nt * BN;
+__device__ __forceinline__ EpiIO epi_io(const Item& it, int half) {
+    EpiIO io{4, half * 128, it.nt * BN + half * 128, -1, -1, -1, -1};
     switch (it.type) {
-        case OP_COND: io.stF = EMAP_C; io.stF_col = col0; break;
-        case OP_IN:
-            io.ldF = EMAP_C; io.ldF_col = col0; io.stF = EMAP_H; io.stF_col = col0;
-            io.stH = EMAP_S; io.stH_col = col0;
+        case OP_COND: io.stF = EMAP_C; break;
+        case OP_IN: io.ldF = EMAP_C; io.stF = EMAP_H; io.stH = EMAP_S; break;
+        case OP_SS:
+        case OP_FSS:
+            io.nch = 2; io.acc0 = half * 64; io.col0 = it.nt * 128 + half * 64;
+            io.ldF = EMAP_H; io.stH = EMAP_U;
             break;
-        case OP_MOD:
-            if (it.nt < P.W / 128) {
-                io.nch = 4; io.ldF = EMAP_H; io.ldF_col = it.nt * 128; io.stH = EMAP_U; io.stH_col = it.nt * 128;
-            } else {
-                io.stH = EMAP_G; io.stH_col = (it.nt - P.W / 128) * BN;
-            }
-            break;
-        case OP_FMOD:
-            io.nch = 4; io.ldF = EMAP_H; io.ldF_col = it.nt * 128; io.stH = EMAP_U; io.stH_col = it.nt * 128;
-            break;
-        case OP_G1: io.stH = EMAP_A; io.stH_col = col0; break;
-        case OP_G2:
-            io.ldF = EMAP_H; io.ldF_col = col0; io.ldH = EMAP_G; io.ldH_col = col0;
-            io.stF = EMAP_H; io.stF_col = col0;
-            break;
+        case OP_GATE: io.stH = EMAP_G0 + (it.gsel - 1); break;
+        case OP_G1: io.stH = EMAP_A; break;
+        case OP_G2: io.ldF = EMAP_H; io.ldH = EMAP_G0 + (it.gsel - 1); io.stF = EMAP_H; break;
         default: io.nch = 0; break;   // OP_OUT: register path
     }
     return io;
@@ -335,70 +378,77 @@ __device__ __forceinline__ void slabH_write(uint32_t base, int r, const float (&
     }
 }
 
+// LayerNorm statistics of one row from its 2*NT partials (mean, M2 over 128 columns each). One pass:
+// the first partial's mean serves as pivot, so nothing cancels.
 __device__ __forceinline__ void row_mean_rstd(const HeadParams& P, int grow, float& mean, float& rstd) {
-    const float2* sp = P.stats + (size_t)grow * P.NT;
-    float msum = 0.f;
-    for (int t = 0; t < P.NT; ++t) msum += ptx::ldcg_f2(sp + t).x;
-    mean = msum / (float)P.NT;
-    float m2 = 0.f;
-    for (int t = 0; t < P.NT; ++t) {
+    const int np = 2 * P.NT;
+    const float2* sp = P.stats + (size_t)grow * np;
+    const float2 v0 = ptx::ldcg_f2(sp);
+    float sd = 0.f, m2 = v0.y;
+#pragma unroll 4
+    for (int t = 1; t < np; ++t) {
         const float2 v = ptx::ldcg_f2(sp + t);
-        const float dm = v.x - mean;
-        m2 += v.y + (float)BN * dm * dm;
+        const float dm = v.x - v0.x;
+        sd += dm;
+        m2 += fmaf(128.0f * dm, dm, v.y);
     }
+    const float dmean = sd / (float)np;                       // mean - pivot
+    mean = v0.x + dmean;
+    m2 = fmaxf(m2 - (float)P.W * dmean * dmean, 0.f);
     rstd = rsqrtf(m2 / (float)P.W + 1e-6f);
 }
 
-// One 32-column chunk of one item. bufF / bufH: this warp's slabs for the chunk; r: lane.
-__device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, int cc, uint32_t tacc,
-                                          uint32_t bufF, uint32_t bufH, int r, Stats& st, float mean,
+// One 32-column chunk of one item. acc: TMEM address of the chunk; col: its global column (bias index
+// for the 256-column ops), bufF / bufH: this warp's slabs for the chunk; r: lane.
+__device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, uint32_t acc, int acc_col, int col,
+                                          bool first, uint32_t bufF, uint32_t bufH, int r, Stats& st, float mean,
                                           float rstd) {
     float v[32];
     switch (it.type) {
         case OP_COND: {                       // c = acc + bc
-            load_acc32(tacc + cc * 32, v);
-            add_bias32(v, P.bc + it.nt * BN + cc * 32);
+            load_acc32(acc, v);
+            add_bias32(v, P.bc + col);
             slabF_write(bufF, r, v);
             break;
         }
         case OP_IN: {                         // h = acc + bin ; s = SiLU(c + temb_k)
-            load_acc32(tacc + cc * 32, v);
-            add_bias32(v, P.bin + it.nt * BN + cc * 32);
-            if (cc == 0) st.init(v[0]);
+            load_acc32(acc, v);
+            add_bias32(v, P.bin + col);
+            if (first) st.init(v[0]);
 #pragma unroll
             for (int i = 0; i < 32; ++i) st.add(v[i]);
             float cv[32];
             slabF_read(bufF, r, cv);
             slabF_write(bufF, r, v);
-            add_bias32(cv, P.temb + (size_t)it.k * P.W + it.nt * BN + cc * 32);
+            add_bias32(cv, P.temb + (size_t)it.k * P.W + col);
 #pragma unroll
             for (int i = 0; i < 32; ++i) cv[i] = silu_f(cv[i]);
             slabH_write(bufH, r, cv);
             break;
         }
-        case OP_MOD:
-        case OP_FMOD: {
-            const float* bias = P.bias_cat + it.b_row;
-            if (it.type == OP_FMOD || it.nt < P.W / 128) {   // u = LN(h) * (1 + scale) + shift
-                float sc[32], hv[32];
-                load_acc32(tacc + cc * 32, v);
-                load_acc32(tacc + 128 + cc * 32, sc);
-                add_bias32(v, bias + cc * 32);
-                add_bias32(sc, bias + 128 + cc * 32);
-                slabF_read(bufF, r, hv);
+        case OP_SS:
+        case OP_FSS: {                        // u = LN(h) * (1 + scale) + shift
+            const float* bias = P.bias_cat + it.b_row + acc_col;
+            float sc[32], hv[32];
+            load_acc32(acc, v);
+            load_acc32(acc + 128, sc);
+            add_bias32(v, bias);
+            add_bias32(sc, bias + 128);
+            slabF_read(bufF, r, hv);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], v[i]);
-                slabH_write(bufH, r, hv);
-            } else {                                          // g = acc + bias
-                load_acc32(tacc + cc * 32, v);
-                add_bias32(v, bias + cc * 32);
-                slabH_write(bufH, r, v);
-            }
+            for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], v[i]);
+            slabH_write(bufH, r, hv);
+            break;
+        }
+        case OP_GATE: {                       // g = acc + bias
+            load_acc32(acc, v);
+            add_bias32(v, P.bias_cat + it.b_row + acc_col);
+            slabH_write(bufH, r, v);
             break;
         }
         case OP_G1: {                         // a = SiLU(acc + b1)
-            load_acc32(tacc + cc * 32, v);
-            add_bias32(v, P.bias_cat + it.b_row + cc * 32);
+            load_acc32(acc, v);
+            add_bias32(v, P.bias_cat + it.b_row + acc_col);
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = silu_f(v[i]);
             slabH_write(bufH, r, v);
@@ -406,13 +456,13 @@ __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, i
         }
         default: {                            // OP_G2: h += g * (acc + b2)
             float gv[32], hv[32];
-            load_acc32(tacc + cc * 32, v);
-            add_bias32(v, P.bias_cat + it.b_row + cc * 32);
+            load_acc32(acc, v);
+            add_bias32(v, P.bias_cat + it.b_row + acc_col);
             slabH_read(bufH, r, gv);
             slabF_read(bufF, r, hv);
 #pragma unroll
             for (int i = 0; i < 32; ++i) hv[i] = fmaf(gv[i], v[i], hv[i]);
-            if (cc == 0) st.init(hv[0]);
+            if (first) st.init(hv[0]);
 #pragma unroll
             for (int i = 0; i < 32; ++i) st.add(hv[i]);
             slabF_write(bufF, r, hv);
@@ -463,11 +513,12 @@ __device__ __forceinline__ void epi_out(const HeadParams& P, const Item& it, uin
     }
 }
 
-// rows of this token tile: z = cond[idx[j]], x = noise[idx[j]], xb = bf16(x); rows past count: 0
-__device__ __forceinline__ void gather_rows(const HeadParams& P, const Item& it, int ewarp, int lane,
-                                            int count) {
+// 16 rows of this token tile per epilogue warp: z = cond[idx[j]], x = noise[idx[j]], xb = bf16(x);
+// rows past count: 0
+__device__ __forceinline__ void gather_rows(const HeadParams& P, const Item& it, int ew, int lane, int count) {
     const int chunks = P.Dc / 8;  // 16-byte chunks per cond row
-    for (int r = ewarp * 32; r < ewarp * 32 + 32; ++r) {
+    constexpr int RPW = BM / EPI_WARPS;
+    for (int r = ew * RPW; r < ew * RPW + RPW; ++r) {
         const int j = it.abs_m * BM + r;
         const int grow = it.slot_row0 + r;
         const bool valid = j < count;
@@ -488,34 +539,30 @@ __device__ __forceinline__ void gather_rows(const HeadParams& P, const Item& it,
 }
 
 // ------------------------------------------------------------------------------------------
-// the persistent kernel. PAIR = false: every CTA works alone (tcgen05 cta_group::1).
-// PAIR = true: clusters of two CTAs; both load their own token tile (A) and half of the weight
-// tile (B); the even CTA issues cta_group::2 MMAs that read both CTAs' shared memory and write
-// 128 accumulator rows into each CTA's TMEM; every CTA runs the epilogue of its own token tile.
+// the persistent kernel: clusters of two CTAs. Both load their own token tile (A) and half of the
+// weight tile (B); the even CTA issues cta_group::2 MMAs that read both CTAs' shared memory and
+// write 128 accumulator rows into each CTA's TMEM; every CTA runs the epilogue of its own token tile.
 // ------------------------------------------------------------------------------------------
-template <bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_constant__ HeadParams P) {
-    constexpr int STAGES = Cfg<PAIR>::STAGES;
-    constexpr int STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = ptx::smem_u32(smem);
     const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;      // 1024-aligned
     const uint32_t bars = epi_base + EPI_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (MAX_STAGES + s); };
-    auto tfull_bar = [&](int b) { return bars + 8u * (2 * MAX_STAGES + b); };
-    auto tempty_bar = [&](int b) { return bars + 8u * (2 * MAX_STAGES + 2 + b); };
-    const uint32_t drain_bar = bars + 8u * (2 * MAX_STAGES + 4);
-    auto epi_bar = [&](int w, int b) { return bars + 8u * (2 * MAX_STAGES + 5 + w * EPI_NB + b); };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+    auto dep_bar = [&](uint32_t i) { return bars + 8u * (2 * STAGES + 5 + (i % DEP_BARS)); };
+    auto epi_bar = [&](int w, int b) { return bars + 8u * (2 * STAGES + 5 + DEP_BARS + w * EPI_NB + b); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + EPI_BYTES + 8 * NUM_BARS);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int rank = PAIR ? (int)ptx::cluster_ctarank() : 0;       // tile of the unit this CTA owns
-    constexpr int UPT = PAIR ? 2 : 1;                              // token tiles per unit
-    const int unit_id = (int)blockIdx.x / UPT;
-    const int n_units = (int)gridDim.x / UPT;
+    const int rank = (int)ptx::cluster_ctarank();                  // token tile of the unit this CTA owns
+    const int unit_id = (int)blockIdx.x / 2;
+    const int n_units = (int)gridDim.x / 2;
 
     int count = __ldg(P.count);
     if (count > P.max_tokens) {
@@ -524,7 +571,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     }
     if (count < 0) count = 0;
     const int MT = (count + BM - 1) / BM;
-    const int MTu = (MT + UPT - 1) / UPT;      // an odd last tile gets an all-padding partner
+    const int MTu = (MT + 1) / 2;                  // an odd last tile gets an all-padding partner
+    const int n_groups = (MTu + P.TGu - 1) / P.TGu;
+    const int tgu = n_groups > 0 ? (MTu + n_groups - 1) / n_groups : 1;   // balanced group size
     const long long total = (long long)MTu * P.T_chain;
 
     if (threadIdx.x == 0) {
@@ -534,75 +583,74 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 4 * UPT);   // epilogue warps of every CTA of the unit
+            ptx::mbar_init(tempty_bar(b), 2 * EPI_WARPS);   // epilogue warps of both CTAs of the unit
         }
         ptx::mbar_init(drain_bar, 1);
-        for (int w = 0; w < 4; ++w)
+        for (int i = 0; i < DEP_BARS; ++i) ptx::mbar_init(dep_bar(i), 1);
+        for (int w = 0; w < EPI_WARPS; ++w)
             for (int b = 0; b < EPI_NB; ++b) ptx::mbar_init(epi_bar(w, b), 1);
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
-        if (PAIR) {
-            ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
-            ptx::tmem_relinquish_pair();
-        } else {
-            ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
-            ptx::tmem_relinquish();
-        }
+        ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
+        ptx::tmem_relinquish_pair();
     }
     ptx::tc_fence_before();
-    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();
+    ptx::cluster_sync_all();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    bool aborted = false;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         int stage = 0;
         uint32_t phase = 0;
         uint32_t issued = 0, issued_parity = 0;
-        for (long long item = unit_id; item < total; item += n_units) {
-            Item it;
-            decode_item(P, MTu, UPT, rank, item, it);
+        uint32_t seq = 0;
+        bool aborted = false;
+        ItemStream ist;
+        Item it;
+        TRACE_DECL
+        while (ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, it)) {
             if (it.type == OP_GATHER) continue;
             bool ok = true;
-            if (lane == 0) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
+            if (lane == 0) {
+                const int* ctr = P.counters + (size_t)it.abs_m * CTRS;
+                ok = wait_counters(ctr, it.needA, it.needB ? ctr + it.gsel : nullptr, it.needB, P);
+            }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { aborted = true; break; }
+            TRACE(0, 0);
+            if (lane == 0) ptx::mbar_arrive(dep_bar(seq));      // the epilogue may now load this item's slabs
+            ++seq;
             ptx::fence_proxy_async();
             const void* map_a = P.maps + it.map_a;
             const void* map_b = P.maps + it.map_b;
-            const int b_rows = it.umma_n / UPT;                       // rows of B this CTA stages
-            const uint32_t tx = (uint32_t)UPT * (A_BYTES + (uint32_t)b_rows * BK * 2);
+            const int b_rows = it.umma_n / 2;                         // rows of B this CTA stages
+            const uint32_t tx = 2u * (A_BYTES + (uint32_t)b_rows * BK * 2);
             for (int kb = 0; kb < it.kblocks; ++kb) {
                 ok = wait_mbar(empty_bar(stage), phase ^ 1u, P);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if (kb == 0) TRACE(0, 1);
                 if (lane == 0) {
                     const uint32_t sa = smem_base + stage * STAGE_BYTES;
-                    if (PAIR) {
-                        // the even CTA arms its barrier for the bytes of both CTAs
-                        if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-                        ptx::tma_load_2d_pair(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
-                        ptx::tma_load_2d_pair(sa + A_BYTES, map_b, full_bar(stage), kb * BK,
-                                              it.b_row + rank * b_rows);
-                    } else {
-                        ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-                        ptx::tma_load_2d(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
-                        ptx::tma_load_2d(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row);
-                    }
+                    // the even CTA arms its barrier for the bytes of both CTAs
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                    ptx::tma_load_2d_pair(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
+                    ptx::tma_load_2d_pair(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row + rank * b_rows);
                 }
                 issued |= 1u << stage;
                 issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
+            TRACE(0, 2); TRACE_TYPE(0); TRACE_NEXT();
             if (!ok) { aborted = true; break; }
         }
-        // own copies in flight must have landed before the CTA exits. Alone (or as the even CTA)
-        // the full barriers are local: wait for every stage's last issue. The odd CTA's loads are
-        // counted on the even CTA's barriers; after a normal run they were all consumed, after an
-        // abort it simply waits out a bounded time that covers any TMA latency.
-        if (!PAIR || rank == 0) {
+        // own copies in flight must have landed before the CTA exits. In the even CTA the full
+        // barriers are local: wait for every stage's last issue. The odd CTA's loads are counted on
+        // the even CTA's barriers; after a normal run they were all consumed, after an abort it
+        // simply waits out a bounded time that covers any TMA latency.
+        if (rank == 0) {
             for (int s = 0; s < STAGES; ++s)
                 if (issued & (1u << s)) wait_mbar(full_bar(s), (issued_parity >> s) & 1u, P, kDrainLimitNs);
         } else if (aborted) {
@@ -610,26 +658,29 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer (the even CTA of a pair issues for both) ----------------
-        if (!PAIR || rank == 0) {
+        // ---------------- MMA issuer (the even CTA issues for the pair) ----------------
+        if (rank == 0) {
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_iter = 0;
-            for (long long item = unit_id; item < total; item += n_units) {
-                Item it;
-                decode_item(P, MTu, UPT, rank, item, it);
+            ItemStream ist;
+            Item it;
+            TRACE_DECL
+            while (ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, it)) {
                 if (it.type == OP_GATHER) continue;
                 const uint32_t buf = acc_iter & 1u;
                 const uint32_t acc_phase = (acc_iter >> 1) & 1u;
                 bool ok = wait_mbar(tempty_bar(buf), acc_phase ^ 1u, P);
                 ok = __all_sync(0xffffffffu, ok);
+                TRACE(1, 0);
                 if (!ok) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                const uint32_t idesc = ptx::idesc_bf16_f32(BM * UPT, (uint32_t)it.umma_n);
+                const uint32_t idesc = ptx::idesc_bf16_f32(2 * BM, (uint32_t)it.umma_n);
                 for (int kb = 0; kb < it.kblocks; ++kb) {
                     ok = wait_mbar(full_bar(stage), phase, P);
                     ok = __all_sync(0xffffffffu, ok);
+                    if (kb == 0) TRACE(1, 1);
                     if (!ok) break;
                     ptx::tc_fence_after();
                     if (lane == 0) {
@@ -637,103 +688,101 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                         const uint64_t da = ptx::smem_desc_sw128(sa);
                         const uint64_t db = ptx::smem_desc_sw128(sa + A_BYTES);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k) {
-                            if (PAIR)
-                                ptx::mma_f16_ss_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
-                                                     (kb | k) != 0 ? 1u : 0u);
-                            else
-                                ptx::mma_f16_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
-                                                (kb | k) != 0 ? 1u : 0u);
-                        }
-                        if (PAIR) ptx::mma_commit_pair_mc(empty_bar(stage), 3);   // frees the stage in both CTAs
-                        else ptx::mma_commit(empty_bar(stage));
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::mma_f16_ss_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
+                                                 (kb | k) != 0 ? 1u : 0u);
+                        ptx::mma_commit_pair_mc(empty_bar(stage), 3);   // frees the stage in both CTAs
                     }
                     __syncwarp();
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if (lane == 0) {
-                    if (PAIR) ptx::mma_commit_pair_mc(tfull_bar(buf), 3);
-                    else ptx::mma_commit(tfull_bar(buf));
-                }
+                if (lane == 0) ptx::mma_commit_pair_mc(tfull_bar(buf), 3);
                 __syncwarp();
                 ++acc_iter;
+                TRACE(1, 2); TRACE_TYPE(1); TRACE_NEXT();
             }
             // all MMAs this thread issued must be done before TMEM is freed
-            if (lane == 0) {
-                if (PAIR) ptx::mma_commit_pair(drain_bar);
-                else ptx::mma_commit(drain_bar);
-            }
+            if (lane == 0) ptx::mma_commit_pair(drain_bar);
             __syncwarp();
             wait_mbar(drain_bar, 0, P, kDrainLimitNs);
         }
     } else {
         // ---------------- epilogue warps ----------------
-        const int ewarp = warp - 2;           // 0..3
+        const int ew = warp - 2;              // 0..7
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
+        const int half = ew >> 2;             // column half of the accumulator this warp takes
         const int row = quarter * 32 + lane;  // row of the tile owned by this thread
-        const bool leader = (threadIdx.x == 64);
-        const uint32_t my_buf = epi_base + (uint32_t)ewarp * EPI_NB * EPI_BUF;
+        const uint32_t my_buf = epi_base + (uint32_t)ew * EPI_NB * EPI_BUF;
         uint32_t ld_parity = 0;               // bit b: parity to wait for on this warp's barrier b
         uint32_t ld_pending = 0;              // bit b: a load into buffer b is in flight
         uint32_t acc_iter = 0;
-        for (long long item = unit_id; item < total; item += n_units) {
-            Item it;
-            decode_item(P, MTu, UPT, rank, item, it);
+        uint32_t seq = 0;
+        ItemStream ist;
+        Item it;
+        TRACE_DECL
+        while (ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, it)) {
             bool fail = false;
             if (it.type == OP_GATHER) {
                 bool ok = true;
-                if (leader && it.abs_m >= P.slots)
-                    ok = wait_counter(P.counters + (it.abs_m - P.slots), P.T_chain, P);
-                if (epi_any(!ok)) break;
-                gather_rows(P, it, ewarp, lane, count);
+                // the scratch slot is free once the token tile that used it before has run its whole chain
+                if (lane == 0 && it.abs_m >= P.slots)
+                    ok = wait_counters(P.counters + (size_t)(it.abs_m - P.slots) * CTRS, EPI_WARPS * P.C_total,
+                                       nullptr, 0, P);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                gather_rows(P, it, ew, lane, count);
             } else {
-                // producers of this token tile first: the chunk loads below read what they wrote
-                bool ok = true;
-                if (leader) ok = wait_counter(P.counters + it.abs_m, it.prior, P);
-                if (epi_any(!ok)) break;
+                // the producer has seen this item's dependencies complete
+                bool ok = wait_mbar(dep_bar(seq), (seq / DEP_BARS) & 1u, P);
+                ok = __all_sync(0xffffffffu, ok);
+                ++seq;
+                if (!ok) break;
+                if (ew == 0) TRACE(2, 0);
                 ptx::fence_proxy_async();
-                const EpiIO io = epi_io(P, it);
+                const EpiIO io = epi_io(it, half);
                 const bool has_loads = (io.ldF >= 0) || (io.ldH >= 0);
                 const int row0 = it.slot_row0 + quarter * 32;
-                auto issue_load = [&](int cc) {
-                    const int b = cc % EPI_NB;
+                auto issue_load = [&](int j) {
+                    const int b = j & 1;
                     if (lane == 0) {
-                        const uint32_t bar = epi_bar(ewarp, b);
+                        const uint32_t bar = epi_bar(ew, b);
                         const uint32_t dst = my_buf + (uint32_t)b * EPI_BUF;
                         ptx::mbar_arrive_expect_tx(bar, (io.ldF >= 0 ? SLAB_F : 0) + (io.ldH >= 0 ? SLAB_H : 0));
-                        if (io.ldF >= 0) ptx::tma_load_2d(dst, P.maps + io.ldF, bar, io.ldF_col + 32 * cc, row0);
-                        if (io.ldH >= 0)
-                            ptx::tma_load_2d(dst + SLAB_F, P.maps + io.ldH, bar, io.ldH_col + 32 * cc, row0);
+                        if (io.ldF >= 0) ptx::tma_load_2d(dst, P.maps + io.ldF, bar, io.col0 + 32 * j, row0);
+                        if (io.ldH >= 0) ptx::tma_load_2d(dst + SLAB_F, P.maps + io.ldH, bar, io.col0 + 32 * j, row0);
                     }
                     ld_pending |= 1u << b;
                 };
-                if (has_loads) {
-                    issue_load(0);
-                    if (io.nch > 1) issue_load(1);
-                }
+                if (has_loads && io.nch > 0) issue_load(0);
+                const int grow = it.slot_row0 + row;
+                float mean = 0.f, rstd = 0.f;
+                if (it.type == OP_SS || it.type == OP_FSS) row_mean_rstd(P, grow, mean, rstd);
                 const uint32_t buf = acc_iter & 1u;
                 const uint32_t acc_phase = (acc_iter >> 1) & 1u;
                 ok = wait_mbar(tfull_bar(buf), acc_phase, P);
                 ok = __all_sync(0xffffffffu, ok);
                 fail = !ok;
+                if (ew == 0) TRACE(2, 1);
                 ptx::tc_fence_after();
                 const uint32_t tacc = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
-                const int grow = it.slot_row0 + row;
                 if (it.type == OP_OUT) {
-                    if (!fail) epi_out(P, it, tacc, grow, it.abs_m * BM + row, count);
+                    if (!fail && half == 0) epi_out(P, it, tacc, grow, it.abs_m * BM + row, count);
                 } else {
                     Stats st;
                     st.init(0.f);
-                    float mean = 0.f, rstd = 0.f;
-                    if (it.type == OP_FMOD || (it.type == OP_MOD && it.nt < P.W / 128)) row_mean_rstd(P, grow, mean, rstd);
 #pragma unroll 1
-                    for (int cc = 0; cc < io.nch; ++cc) {
-                        const int b = cc % EPI_NB;
+                    for (int j = 0; j < io.nch; ++j) {
+                        const int b = j & 1;
                         const uint32_t bufF = my_buf + (uint32_t)b * EPI_BUF;
                         const uint32_t bufH = bufF + SLAB_F;
                         if (has_loads) {
-                            bool okw = wait_mbar(epi_bar(ewarp, b), (ld_parity >> b) & 1u, P);
+                            if (j + 1 < io.nch) {
+                                // the other buffer was the source of the previous chunk's store
+                                if (lane == 0) ptx::bulk_wait_read<0>();
+                                issue_load(j + 1);
+                            }
+                            bool okw = wait_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u, P);
                             okw = __all_sync(0xffffffffu, okw);
                             ld_parity ^= 1u << b;
                             ld_pending &= ~(1u << b);
@@ -743,53 +792,51 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                             if (lane == 0) ptx::bulk_wait_read<EPI_NB - 1>();
                             __syncwarp();
                         }
-                        epi_chunk(P, it, cc, tacc, bufF, bufH, lane, st, mean, rstd);
+                        epi_chunk(P, it, tacc + io.acc0 + 32 * j, io.acc0 + 32 * j, io.col0 + 32 * j, j == 0, bufF, bufH,
+                                  lane, st, mean, rstd);
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
-                        if (has_loads && cc + 2 < io.nch) {
-                            // buffer of chunk cc+2 = buffer of chunk cc-1: its store must be done reading
-                            if (lane == 0) ptx::bulk_wait_read<0>();
-                            issue_load(cc + 2);
-                        }
                         if (lane == 0) {
-                            if (io.stF >= 0) ptx::tma_store_2d(P.maps + io.stF, bufF, io.stF_col + 32 * cc, row0);
-                            if (io.stH >= 0) ptx::tma_store_2d(P.maps + io.stH, bufH, io.stH_col + 32 * cc, row0);
+                            if (io.stF >= 0) ptx::tma_store_2d(P.maps + io.stF, bufF, io.col0 + 32 * j, row0);
+                            if (io.stH >= 0) ptx::tma_store_2d(P.maps + io.stH, bufH, io.col0 + 32 * j, row0);
                             ptx::bulk_commit();
                         }
                     }
-                    if (it.type == OP_IN || it.type == OP_G2) P.stats[(size_t)grow * P.NT + it.nt] = st.finish(BN);
+                    if (it.type == OP_IN || it.type == OP_G2)
+                        P.stats[(size_t)grow * (2 * P.NT) + it.nt * 2 + half] = st.finish(128);
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
-                    if (PAIR) ptx::mbar_arrive_even_cta(tempty_bar(buf));
-                    else ptx::mbar_arrive(tempty_bar(buf));
-                }
+                if (lane == 0) ptx::mbar_arrive_even_cta(tempty_bar(buf));
                 ++acc_iter;
                 if (lane == 0) ptx::bulk_wait<0>();   // this warp's stores are performed
                 __syncwarp();
             }
-            // publish: this item's global writes, then one tick of the token tile's counter
+            if (fail) break;
+            // publish: this warp's global writes, then one tick of the token tile's counter
             __threadfence();
             ptx::fence_proxy_async();
-            const bool any_fail = epi_any(fail);
-            if (any_fail) break;
-            if (leader) ptx::red_release_gpu_add(P.counters + it.abs_m, 1);
+            __syncwarp();
+            if (lane == 0)
+                ptx::red_release_gpu_add(P.counters + (size_t)it.abs_m * CTRS + (it.type == OP_GATE ? it.gsel : 0), 1);
+            if (it.type != OP_GATHER) {
+                if (ew == 0) { TRACE(2, 2); TRACE_TYPE(2); }
+                TRACE_NEXT();
+            }
         }
         // own copies in flight: loads that were issued but never consumed, stores not yet done
         for (int b = 0; b < EPI_NB; ++b)
-            if (ld_pending & (1u << b)) wait_mbar(epi_bar(ewarp, b), (ld_parity >> b) & 1u, P, kDrainLimitNs);
+            if (ld_pending & (1u << b)) wait_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u, P, kDrainLimitNs);
         if (lane == 0) ptx::bulk_wait<0>();
         __syncwarp();
     }
 
     ptx::tc_fence_before();
     // nobody leaves while its partner may still signal its barriers or read its shared memory
-    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();
+    ptx::cluster_sync_all();
     if (warp == 1) {
         ptx::tc_fence_after();
-        if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512);
-        else ptx::tmem_dealloc(tmem_base, 512);
+        ptx::tmem_dealloc_pair(tmem_base, 512);
     }
 }
 
@@ -925,18 +972,20 @@ inline float bf16_bits_to_float(uint16_t b) {
 
 struct ardiff_head {
     ardiff_head_desc d;
-    int device, n_sm, grid, pair, coop;
-    int NT, TG, slots, T_pro, T_step, T_chain, n_step_ops;
+    int device, n_sm, grid, coop;
+    int NT, TGu, slots, T_pro, T_step, C_pro, C_step, gcnt[2], n_phases;
     int64_t max_tiles;
     std::vector<void*> allocs;
     // device
     bf16 *Wcat, *Wc, *Win, *Wt1, *Wt2;
     float *bias_cat, *bc, *bin, *bt1, *bt2, *temb, *temb_hidden;
-    bf16 *z, *xb, *s, *u, *a, *g;
+    bf16 *z, *xb, *s, *u, *a, *g0, *g1;
     float *x, *c, *h;
     float2* stats;
     int *counters, *status;  // status[0] = status word, status[1] = abort flag
-    StepOp* step_ops;
+    long long* trace;        // per-item time stamps (only with ARDIFF_HEAD_PROFILE)
+    Phase* phases;
+    uint16_t* cum2phase;
     CUtensorMap* maps;
     // optional timing of the persistent kernel
     int timing, timed;
@@ -1017,64 +1066,57 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     H->device = dev;
     H->n_sm = prop.multiProcessorCount;
     const int W = d.W, C = d.C, Dc = d.Dc, L = d.L;
-    H->NT = W / BN;
-    H->T_pro = 1 + H->NT;
-    H->T_step = H->NT * (3 + 5 * L) + 1;
-    H->n_step_ops = 3 * L + 3;
+    const int NT = W / BN;
+    H->NT = NT;
+    H->T_pro = 1 + NT;
+    H->T_step = NT * (3 + 5 * L) + 1;
+    H->C_pro = 1 + NT;
+    H->C_step = NT * (3 + 4 * L) + 1;
+    H->gcnt[0] = NT * ((L + 1) / 2);
+    H->gcnt[1] = NT * (L / 2);
     H->max_tiles = (d.max_tokens + BM - 1) / BM;
     if (H->max_tiles < 1) H->max_tiles = 1;
 
-    // grid: one CTA per SM, all co-resident (cooperative launch). Default: CTA pairs (clusters of 2).
-    H->pair = env_int("ARDIFF_HEAD_PAIR", 1) != 0;
+    // grid: one CTA per SM in clusters of two, all co-resident.
     // The cooperative attribute makes the launch fail instead of start when the grid cannot be
     // co-resident. ARDIFF_HEAD_COOP=0 drops it for tools that cannot replay such launches (the
     // grid is still sized to be co-resident on an otherwise idle device, and every wait is bounded).
     H->coop = env_int("ARDIFF_HEAD_COOP", 1) != 0;
-    {
-        bool ok = cudaFuncSetAttribute(head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       smem_bytes<false>()) == cudaSuccess;
-        ok &= cudaFuncSetAttribute(head_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   smem_bytes<true>()) == cudaSuccess;
-        int per_sm = 0;
-        ok = ok && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, head_kernel<false>, NUM_THREADS,
-                                                                 smem_bytes<false>()) == cudaSuccess && per_sm >= 1;
-        if (!ok) {
-            (void)cudaGetLastError();
-            delete H;
-            return ARDIFF_ERR_CUDA;
-        }
-    }
     H->grid = env_int("ARDIFF_HEAD_GRID", H->n_sm);
-    if (H->grid < 1 || H->grid > H->n_sm) H->grid = H->n_sm;
-    if (H->pair) {
-        // every cluster of two must be resident at once
+    if (H->grid < 2 || H->grid > H->n_sm) H->grid = H->n_sm;
+    H->grid &= ~1;
+    {
+        bool ok = cudaFuncSetAttribute(head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) ==
+                  cudaSuccess;
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-        cfg.gridDim = dim3(H->grid & ~1); cfg.blockDim = dim3(NUM_THREADS);
-        cfg.dynamicSmemBytes = smem_bytes<true>(); cfg.attrs = at; cfg.numAttrs = 1;
+        cfg.gridDim = dim3(H->grid); cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = SMEM_BYTES; cfg.attrs = at; cfg.numAttrs = 1;
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, head_kernel<true>, &cfg) != cudaSuccess || max_clusters < 1) {
+        ok = ok && cudaOccupancyMaxActiveClusters(&max_clusters, head_kernel, &cfg) == cudaSuccess && max_clusters >= 1;
+        if (!ok) {
             (void)cudaGetLastError();
-            H->pair = 0;
-        } else {
-            H->grid &= ~1;
-            if (H->grid > 2 * max_clusters) H->grid = 2 * max_clusters;
+            delete H;
+            return ARDIFF_ERR_CUDA;
         }
+        if (H->grid > 2 * max_clusters) H->grid = 2 * max_clusters;
     }
-    const int units = H->pair ? H->grid / 2 : H->grid;
+    const int units = H->grid / 2;
 
-    // token tiles per group: enough column tiles per layer to keep every unit busy while the
-    // layer before it drains (about 1.5 grids of items), capped by what exists
-    int tg = ((3 * units / 2 + H->NT - 1) / H->NT) * (H->pair ? 2 : 1);
-    tg = env_int("ARDIFF_HEAD_TG", tg);
-    if (tg < 1) tg = 1;
-    if ((int64_t)tg > H->max_tiles) tg = (int)H->max_tiles;
-    if (H->pair) tg = (tg + 1) & ~1;
-    H->TG = tg;
-    H->slots = 2 * tg;
+    // largest group, in units (pairs of token tiles): a phase of NT column tiles per token tile should
+    // span about 2.5 grids of items so that a dependent phase finds its producers long finished
+    int tgu = (5 * units / 2 + NT - 1) / NT;
+    {
+        const int tg_env = env_int("ARDIFF_HEAD_TGU", 0);
+        if (tg_env > 0) tgu = tg_env;
+    }
+    if (tgu < 1) tgu = 1;
+    if ((int64_t)tgu * 2 > H->max_tiles + 1) tgu = (int)((H->max_tiles + 1) / 2);
+    H->TGu = tgu;
+    H->slots = 4 * tgu;   // two groups of token tiles
     const size_t R = (size_t)H->slots * BM;
 
     // ---- pack the weights: one K-major matrix [rows][W] for every W-input layer ----
@@ -1139,41 +1181,59 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     TRY(dev_alloc(H, &H->s, R * W, true));
     TRY(dev_alloc(H, &H->u, R * W, true));
     TRY(dev_alloc(H, &H->a, R * W, true));
-    TRY(dev_alloc(H, &H->g, R * W, true));
+    TRY(dev_alloc(H, &H->g0, R * W, true));
+    TRY(dev_alloc(H, &H->g1, R * W, true));
     TRY(dev_alloc(H, &H->x, R * C, true));
     TRY(dev_alloc(H, &H->c, R * W, true));
     TRY(dev_alloc(H, &H->h, R * W, true));
-    TRY(dev_alloc(H, &H->stats, R * H->NT, true));
-    TRY(dev_alloc(H, &H->counters, (size_t)H->max_tiles + 2, true));
+    TRY(dev_alloc(H, &H->stats, R * 2 * NT, true));
+    TRY(dev_alloc(H, &H->counters, ((size_t)H->max_tiles + 2) * CTRS, true));
     TRY(dev_alloc(H, &H->status, 2, true));
+#ifdef ARDIFF_HEAD_PROFILE
+    TRY(dev_alloc(H, &H->trace, (size_t)TRACE_ITEMS * 3 * 4, true));
+#endif
 
-    // ---- op table of one step ----
+    // ---- the program of one step: phases in list order ----
     {
-        std::vector<StepOp> ops;
+        std::vector<Phase> ph;
         int cum = 0;
-        auto add = [&](int type, int ntiles, int ma, int mb, size_t b_row0, int kblocks, int umma_n, int blk) {
-            StepOp o{type, ntiles, cum, ma, mb, (int)b_row0, kblocks, umma_n, blk};
-            ops.push_back(o);
+        auto add = [&](int type, int block, int tile0, int ntiles, size_t b_row0, int offA, int gsel, int goff) {
+            if (ntiles <= 0) return;
+            ph.push_back(Phase{type, block, tile0, ntiles, cum, (int)b_row0, offA, gsel, goff});
             cum += ntiles;
         };
-        const int NT = H->NT, kW = W / BK;
-        add(OP_IN, NT, MAP_XB, MAP_WIN, 0, 1, BN, -1);
+        auto gate = [&](int b, int tile0, int ntiles) {
+            // needs s of this step (the in-projection items) and its buffer, last read by block b-2
+            const int offA = NT + (b >= 2 ? 4 * NT * (b - 1) : 0);
+            add(OP_GATE, b, tile0, ntiles, b * blk_rows + 2 * (size_t)W, offA, 1 + (b & 1), 0);
+        };
+        const int na = NT / 2;   // gate tiles of the next block placed between G1 and G2; the rest follow G2
+        add(OP_IN, -1, 0, NT, 0, 0, 0, 0);
+        gate(0, 0, NT);
         for (int b = 0; b < L; ++b) {
-            add(OP_MOD, 3 * NT, MAP_S, MAP_WCAT, b * blk_rows, kW, BN, b);
-            add(OP_G1, NT, MAP_U, MAP_WCAT, b * blk_rows + 3 * (size_t)W, kW, BN, b);
-            add(OP_G2, NT, MAP_A, MAP_WCAT, b * blk_rows + 4 * (size_t)W, kW, BN, b);
+            const int base = NT + 4 * NT * b;
+            add(OP_SS, b, 0, 2 * NT, b * blk_rows, base, 0, 0);
+            add(OP_G1, b, 0, NT, b * blk_rows + 3 * (size_t)W, base + 2 * NT, 0, 0);
+            if (b + 1 < L) gate(b + 1, 0, na);
+            add(OP_G2, b, 0, NT, b * blk_rows + 4 * (size_t)W, base + 3 * NT, 1 + (b & 1), NT * ((b >> 1) + 1));
+            if (b + 1 < L) gate(b + 1, na, NT - na);
         }
-        add(OP_FMOD, 2 * NT, MAP_S, MAP_WCAT, fm_row0, kW, BN, -1);
-        add(OP_OUT, 1, MAP_U, MAP_WOUT, out_row0, kW, C, -1);
-        if (cum != H->T_step || (int)ops.size() != H->n_step_ops) {
+        add(OP_FSS, -1, 0, 2 * NT, fm_row0, NT + 4 * NT * L, 0, 0);
+        add(OP_OUT, -1, 0, 1, out_row0, NT + 4 * NT * L + 2 * NT, 0, 0);
+        if (cum != H->T_step) {
             free_all(H);
             delete H;
             return ARDIFF_ERR_UNSUPPORTED;
         }
-        TRY(dev_alloc(H, &H->step_ops, ops.size(), false));
-        TRY(upload(H->step_ops, ops.data(), ops.size() * sizeof(StepOp)));
+        std::vector<uint16_t> c2p(cum);
+        for (size_t i = 0; i < ph.size(); ++i)
+            for (int t = 0; t < ph[i].ntiles; ++t) c2p[ph[i].cum + t] = (uint16_t)i;
+        H->n_phases = (int)ph.size();
+        TRY(dev_alloc(H, &H->phases, ph.size(), false));
+        TRY(upload(H->phases, ph.data(), ph.size() * sizeof(Phase)));
+        TRY(dev_alloc(H, &H->cum2phase, c2p.size(), false));
+        TRY(upload(H->cum2phase, c2p.data(), c2p.size() * sizeof(uint16_t)));
     }
-    H->T_chain = H->T_pro + d.K_max * H->T_step;  // recomputed per call for the call's K
 
     // ---- tensor maps ----
     {
@@ -1184,17 +1244,18 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         ok &= make_map(&maps[MAP_S], H->s, R, W, BM);
         ok &= make_map(&maps[MAP_U], H->u, R, W, BM);
         ok &= make_map(&maps[MAP_A], H->a, R, W, BM);
-        const uint32_t bdiv = H->pair ? 2 : 1;   // a CTA of a pair stages half of the weight tile's rows
-        ok &= make_map(&maps[MAP_WC], H->Wc, W, Dc, BN / bdiv);
-        ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, BN / bdiv);
-        ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, BN / bdiv);
-        ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C / bdiv);
+        // a CTA of a pair stages half of the weight tile's rows
+        ok &= make_map(&maps[MAP_WC], H->Wc, W, Dc, B_ROWS);
+        ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, B_ROWS);
+        ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, B_ROWS);
+        ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C / 2);
         ok &= make_slab_map(&maps[EMAP_H], H->h, R, W, true);
         ok &= make_slab_map(&maps[EMAP_C], H->c, R, W, true);
         ok &= make_slab_map(&maps[EMAP_S], H->s, R, W, false);
         ok &= make_slab_map(&maps[EMAP_U], H->u, R, W, false);
         ok &= make_slab_map(&maps[EMAP_A], H->a, R, W, false);
-        ok &= make_slab_map(&maps[EMAP_G], H->g, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_G0], H->g0, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_G1], H->g1, R, W, false);
         if (!ok) {
             free_all(H);
             delete H;
@@ -1250,20 +1311,24 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
                                                                                   H->temb_hidden);
     temb_out_kernel<<<dim3((W + 7) / 8, K), 256, 0, st>>>(H->Wt2, H->bt2, W, H->temb_hidden, H->temb);
     launches += 2;
-    if (cudaMemsetAsync(H->counters, 0, sizeof(int) * ((size_t)H->max_tiles + 2), st) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    if (cudaMemsetAsync(H->counters, 0, sizeof(int) * ((size_t)H->max_tiles + 2) * CTRS, st) != cudaSuccess)
+        return ARDIFF_ERR_CUDA;
     if (cudaMemsetAsync(H->status + 1, 0, sizeof(int), st) != cudaSuccess) return ARDIFF_ERR_CUDA;
 
     HeadParams P;
     memset(&P, 0, sizeof(P));
-    P.C = C; P.Dc = H->d.Dc; P.W = W; P.L = H->d.L; P.K = K; P.NT = H->NT; P.TG = H->TG; P.slots = H->slots;
-    P.T_pro = H->T_pro; P.T_step = H->T_step; P.T_chain = H->T_pro + K * H->T_step; P.n_step_ops = H->n_step_ops;
+    P.C = C; P.Dc = H->d.Dc; P.W = W; P.L = H->d.L; P.K = K; P.NT = H->NT; P.TGu = H->TGu; P.slots = H->slots;
+    P.T_pro = H->T_pro; P.T_step = H->T_step; P.T_chain = H->T_pro + K * H->T_step;
+    P.C_pro = H->C_pro; P.C_step = H->C_step; P.C_total = H->C_pro + K * H->C_step;
+    P.gcnt[0] = H->gcnt[0]; P.gcnt[1] = H->gcnt[1];
     P.max_tokens = (int)H->d.max_tokens;
-    P.step_ops = H->step_ops; P.maps = H->maps;
+    P.phases = H->phases; P.cum2phase = H->cum2phase; P.maps = H->maps;
     P.cond = reinterpret_cast<const bf16*>(cond); P.noise = noise; P.idx = idx; P.count = count; P.out = out;
-    P.z = H->z; P.xb = H->xb; P.s = H->s; P.u = H->u; P.a = H->a; P.g = H->g;
+    P.z = H->z; P.xb = H->xb; P.s = H->s; P.u = H->u; P.a = H->a; P.g0 = H->g0; P.g1 = H->g1;
     P.x = H->x; P.c = H->c; P.h = H->h; P.stats = H->stats;
     P.bias_cat = H->bias_cat; P.bc = H->bc; P.bin = H->bin; P.temb = H->temb;
     P.counters = H->counters; P.status = H->status; P.abort_flag = H->status + 1;
+    P.trace = H->trace;
     for (int k = 0; k < K; ++k) P.dt[k] = (float)((double)t_sched[k + 1] - (double)t_sched[k]);
 
     ardiff_head* Hm = const_cast<ardiff_head*>(H);
@@ -1278,17 +1343,13 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
             at[na].val.cooperative = 1;
             ++na;
         }
-        if (H->pair) {
-            at[na].id = cudaLaunchAttributeClusterDimension;
-            at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
-            ++na;
-        }
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+        ++na;
         cfg.gridDim = dim3(H->grid); cfg.blockDim = dim3(NUM_THREADS);
-        cfg.dynamicSmemBytes = H->pair ? smem_bytes<true>() : smem_bytes<false>();
+        cfg.dynamicSmemBytes = SMEM_BYTES;
         cfg.stream = st; cfg.attrs = at; cfg.numAttrs = na;
-        cudaError_t e = H->pair ? cudaLaunchKernelEx(&cfg, head_kernel<true>, P)
-                                : cudaLaunchKernelEx(&cfg, head_kernel<false>, P);
-        if (e != cudaSuccess) {
+        if (cudaLaunchKernelEx(&cfg, head_kernel, P) != cudaSuccess) {
             (void)cudaGetLastError();
             return ARDIFF_ERR_CUDA;
         }
@@ -1330,7 +1391,7 @@ extern "C" int ardiff_head_status(ardiff_head* H, void* stream) {
 }
 
 // Internal (not part of the public header): device pointers of the head's scratch arrays, for
-// bring-up scripts that compare intermediates. name: z xb s u a g x c h temb
+// bring-up scripts that compare intermediates. name: z xb s u a g0 g1 x c h temb counters trace
 extern "C" void* ardiff_head_debug_ptr(ardiff_head* H, const char* name) {
     if (!H || !name) return nullptr;
     if (!strcmp(name, "z")) return H->z;
@@ -1338,12 +1399,14 @@ extern "C" void* ardiff_head_debug_ptr(ardiff_head* H, const char* name) {
     if (!strcmp(name, "s")) return H->s;
     if (!strcmp(name, "u")) return H->u;
     if (!strcmp(name, "a")) return H->a;
-    if (!strcmp(name, "g")) return H->g;
+    if (!strcmp(name, "g0")) return H->g0;
+    if (!strcmp(name, "g1")) return H->g1;
     if (!strcmp(name, "x")) return H->x;
     if (!strcmp(name, "c")) return H->c;
     if (!strcmp(name, "h")) return H->h;
     if (!strcmp(name, "temb")) return H->temb;
     if (!strcmp(name, "counters")) return H->counters;
+    if (!strcmp(name, "trace")) return H->trace;
     return nullptr;
 }
 
