@@ -51,9 +51,14 @@ def _load():
         lib.oracle_entropy.argtypes = [vp, i64, i32, vp]
         lib.oracle_gate.argtypes = [vp, i64, i32, ctypes.c_float, vp, vp, vp, vp]
         lib.oracle_head_sample.argtypes = [ctypes.POINTER(_HeadParams), vp, vp, vp, i32, vp, i32, vp]
+        lib.oracle_head_sample_coef.argtypes = [ctypes.POINTER(_HeadParams), vp, vp, vp, i32, vp, vp, i64, vp, i32, vp]
+        lib.oracle_gate_blocks.argtypes = [vp, i64, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp]
+        lib.oracle_tau_calibrate.argtypes = [vp, i64, vp, vp, vp]
+        lib.oracle_accept_prefix.argtypes = [vp, vp, i64, i32, vp]
         lib.oracle_layer_norm.argtypes = [vp, i32, vp]
         lib.oracle_time_embedding.argtypes = [ctypes.POINTER(_HeadParams), ctypes.c_float, vp]
-        for f in (lib.oracle_entropy, lib.oracle_gate, lib.oracle_head_sample,
+        for f in (lib.oracle_entropy, lib.oracle_gate, lib.oracle_head_sample, lib.oracle_head_sample_coef,
+                  lib.oracle_gate_blocks, lib.oracle_tau_calibrate, lib.oracle_accept_prefix,
                   lib.oracle_layer_norm, lib.oracle_time_embedding):
             f.restype = None
         _lib = lib
@@ -131,6 +136,72 @@ def head_sample(weights: Dict[str, np.ndarray], cond_bits: np.ndarray, noise: np
                                t_sched.ctypes.data, K, idx.ctypes.data, idx.shape[0], out.ctypes.data)
     del keep
     return out
+
+
+def head_sample_coef(weights: Dict[str, np.ndarray], cond_bits: np.ndarray, noise: np.ndarray,
+                     t_in: np.ndarray, coef: np.ndarray, idx: np.ndarray,
+                     step_noise: Optional[np.ndarray] = None) -> np.ndarray:
+    """K = len(t_in) head evaluations at times t_in, each followed by x <- ax x + av v + an z_k.
+
+    coef: float32 [K, 3] = (ax, av, an) per step; step_noise: float32 [K, n, C] or None.
+    Returns out [n, C] float64 (rows not in idx are zero)."""
+    p, keep = _params(weights)
+    cond_bits = _u16(cond_bits)
+    noise = np.ascontiguousarray(noise, dtype=np.float32)
+    t_in = np.ascontiguousarray(t_in, dtype=np.float32)
+    coef = np.ascontiguousarray(coef, dtype=np.float32)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    n = noise.shape[0]
+    K = t_in.shape[0]
+    assert coef.shape == (K, 3)
+    sn = None
+    if step_noise is not None:
+        sn = np.ascontiguousarray(step_noise, dtype=np.float32)
+        assert sn.shape == (K, n, p.C)
+    out = np.zeros((n, p.C), dtype=np.float64)
+    _load().oracle_head_sample_coef(ctypes.byref(p), cond_bits.ctypes.data, noise.ctypes.data, t_in.ctypes.data, K,
+                                    coef.ctypes.data, sn.ctypes.data if sn is not None else None, n,
+                                    idx.ctypes.data, idx.shape[0], out.ctypes.data)
+    del keep
+    return out
+
+
+def gate_blocks(feat_bits: np.ndarray, rows_per_token: int, gamma: int, tau: float):
+    """Block-prefix gate (Algorithm 1, Step 1). feat: bf16 bits [n * rows_per_token, d].
+
+    Returns (Hs [n] f64 token indicators, mask [n] u8, idx [count] i32, count, len [ceil(n/gamma)] i32)."""
+    feat_bits = _u16(feat_bits)
+    rows, d = feat_bits.shape
+    assert rows % rows_per_token == 0 and gamma >= 1
+    n = rows // rows_per_token
+    nb = (n + gamma - 1) // gamma
+    Hs = np.empty((n,), dtype=np.float64)
+    mask = np.empty((n,), dtype=np.uint8)
+    idx = np.empty((max(n, 1),), dtype=np.int32)
+    ln = np.empty((max(nb, 1),), dtype=np.int32)
+    count = ctypes.c_int32(0)
+    _load().oracle_gate_blocks(feat_bits.ctypes.data, n, rows_per_token, d, gamma, ctypes.c_float(np.float32(tau)),
+                               Hs.ctypes.data, mask.ctypes.data, idx.ctypes.data, ctypes.byref(count), ln.ctypes.data)
+    return Hs, mask, idx[:count.value].copy(), int(count.value), ln[:nb].copy()
+
+
+def tau_calibrate(H: np.ndarray) -> Tuple[float, float, float]:
+    """(mean, std, tau = 0.3 mean - 0.1 std) of a set of entropies (std with divisor n)."""
+    H = np.ascontiguousarray(H, dtype=np.float64)
+    m, s, t = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    _load().oracle_tau_calibrate(H.ctypes.data, H.shape[0], ctypes.byref(m), ctypes.byref(s), ctypes.byref(t))
+    return m.value, s.value, t.value
+
+
+def accept_prefix(r: np.ndarray, ratio: np.ndarray, gamma: int) -> np.ndarray:
+    """Accepted draft length per block of gamma: first position whose r exceeds its ratio, else the block length."""
+    r = np.ascontiguousarray(r, dtype=np.float32)
+    ratio = np.ascontiguousarray(ratio, dtype=np.float32)
+    n = r.shape[0]
+    nb = (n + gamma - 1) // gamma
+    out = np.empty((max(nb, 1),), dtype=np.int32)
+    _load().oracle_accept_prefix(r.ctypes.data, ratio.ctypes.data, n, gamma, out.ctypes.data)
+    return out[:nb].copy()
 
 
 def layer_norm(h: np.ndarray) -> np.ndarray:

@@ -81,6 +81,67 @@ void oracle_gate(const uint16_t* feat, int64_t n, int32_t d, float tau, double* 
     if (!H) free(Hloc);
 }
 
+/*
+ * Block-prefix gate: the early stop of Algorithm 1, Step 1, as it is written. Token i owns the
+ * r consecutive rows i*r .. i*r+r-1 of feat; its indicator is the mean of their row entropies
+ * (H^s = -L_entropy, the mean over the R rows -- and heads -- of the entropy-loss equation).
+ * Tokens come in draft blocks of gamma (the last block may be shorter). Scanning a block in
+ * order, the first token with H^s < tau ends speculation: it and every later token of the block
+ * are dropped ("draft_tokens[1 : i-1]", "break"). len[b] = tokens kept in block b.
+ */
+void oracle_gate_blocks(const uint16_t* feat, int64_t n, int32_t r, int32_t d, int32_t gamma, float tau,
+                        double* Hs, uint8_t* mask, int32_t* idx, int32_t* count, int32_t* len) {
+    double* Hrow = (double*)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1) * (size_t)r);
+    oracle_entropy(feat, n * r, d, Hrow);
+    for (int64_t i = 0; i < n; ++i) {
+        double acc = 0.0;
+        for (int32_t j = 0; j < r; ++j) acc += Hrow[(size_t)i * (size_t)r + (size_t)j];
+        Hs[i] = acc / (double)r;
+    }
+    free(Hrow);
+    const double t = (double)tau;
+    int32_t k = 0;
+    for (int64_t b0 = 0, b = 0; b0 < n; b0 += gamma, ++b) {
+        const int64_t b1 = (b0 + gamma < n) ? b0 + gamma : n;
+        int speculate = 1;
+        int32_t kept = 0;
+        for (int64_t i = b0; i < b1; ++i) {
+            if (speculate && !(Hs[i] >= t)) speculate = 0; /* H < tau, or NaN */
+            mask[i] = (uint8_t)speculate;
+            if (speculate) { idx[k++] = (int32_t)i; ++kept; }
+        }
+        len[b] = kept;
+    }
+    *count = k;
+}
+
+/* Threshold from entropy statistics ("Entropy-Based Early Stopping", the tau equation):
+ * tau = 0.3 * mean(H) - 0.1 * std(H), std taken over the whole set (divisor n). */
+void oracle_tau_calibrate(const double* H, int64_t n, double* mean, double* std, double* tau) {
+    double m = 0.0;
+    for (int64_t i = 0; i < n; ++i) m += H[i];
+    m /= (double)n;
+    double v = 0.0;
+    for (int64_t i = 0; i < n; ++i) v += (H[i] - m) * (H[i] - m);
+    v /= (double)n;
+    *mean = m;
+    *std = sqrt(v);
+    *tau = 0.3 * m - 0.1 * sqrt(v);
+}
+
+/* Accepted draft length per block (Algorithm 1, Step 4):
+ * n_b = min({i-1 : r_i > ratio_i} U {len_b}), i counted from 1 inside the block. */
+void oracle_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma, int32_t* nacc) {
+    for (int64_t b0 = 0, b = 0; b0 < n; b0 += gamma, ++b) {
+        const int64_t b1 = (b0 + gamma < n) ? b0 + gamma : n;
+        int32_t acc = (int32_t)(b1 - b0);
+        for (int64_t i = b0; i < b1; ++i) {
+            if (r[i] > ratio[i]) { acc = (int32_t)(i - b0); break; }
+        }
+        nacc[b] = acc;
+    }
+}
+
 /* ------------------------------------------------------------------------------------
  * Head.  All parameters are bf16 bit patterns widened exactly to double; noise and the
  * time schedule are float32 widened to double; nothing is rounded in between.
@@ -139,8 +200,12 @@ static void time_embedding(const oracle_head_params* P, double t, double* temb, 
 }
 
 /* One survivor token: K Euler steps of the velocity head. x [C] in/out. */
+/* One survivor token: K steps of the head, each followed by the sampler update
+ *   x <- ax_k x + av_k v + an_k z_k        (coef = {ax_0, av_0, an_0, ax_1, ...}, z_k = step noise or none).
+ * The Euler flow update is the case ax = 1, av = t_{k+1} - t_k, an = 0. */
 static void head_token(const oracle_head_params* P, const uint16_t* z_bits, const double* temb_all,
-                       const float* t_sched, int32_t K, double* x, double* buf) {
+                       const double* coef, const float* step_noise_tok, size_t step_stride, int32_t K, double* x,
+                       double* buf) {
     const int32_t C = P->C, Dc = P->Dc, W = P->W, L = P->L;
     double* z = buf;              /* Dc */
     double* c = z + Dc;           /* W  */
@@ -171,8 +236,12 @@ static void head_token(const oracle_head_params* P, const uint16_t* z_bits, cons
         layer_norm(h, W, u);
         for (int32_t i = 0; i < W; ++i) u[i] = u[i] * (1.0 + mod[W + i]) + mod[i];
         linear(P->Wout, P->bout, C, W, u, v);
-        const double dt = (double)t_sched[k + 1] - (double)t_sched[k];
-        for (int32_t i = 0; i < C; ++i) x[i] += dt * v[i];
+        const double ax = coef[3 * k], av = coef[3 * k + 1], an = coef[3 * k + 2];
+        for (int32_t i = 0; i < C; ++i) {
+            double xn = ax * x[i] + av * v[i];
+            if (step_noise_tok) xn += an * (double)step_noise_tok[(size_t)k * step_stride + (size_t)i];
+            x[i] = xn;
+        }
     }
 }
 
@@ -181,9 +250,9 @@ static void head_token(const oracle_head_params* P, const uint16_t* z_bits, cons
  * idx [count] token ids (any order), out [n][C] double: only rows idx[j] are written.
  * K = 0 copies the noise rows.
  */
-void oracle_head_sample(const oracle_head_params* P, const uint16_t* cond, const float* noise,
-                        const float* t_sched, int32_t K, const int32_t* idx, int32_t count,
-                        double* out) {
+static void head_sample_coef(const oracle_head_params* P, const uint16_t* cond, const float* noise,
+                             const float* t_sched, int32_t K, const double* coef, const float* step_noise,
+                             int64_t n, const int32_t* idx, int32_t count, double* out) {
     const int32_t C = P->C, Dc = P->Dc, W = P->W;
     double* temb_all = (double*)malloc(sizeof(double) * (size_t)(K > 0 ? K : 1) * (size_t)W);
     {
@@ -203,11 +272,42 @@ void oracle_head_sample(const oracle_head_params* P, const uint16_t* cond, const
             const size_t tok = (size_t)idx[j];
             double* x = out + tok * (size_t)C;
             for (int32_t i = 0; i < C; ++i) x[i] = (double)noise[tok * (size_t)C + i];
-            head_token(P, cond + tok * (size_t)Dc, temb_all, t_sched, K, x, buf);
+            head_token(P, cond + tok * (size_t)Dc, temb_all, coef,
+                       step_noise ? step_noise + tok * (size_t)C : NULL, (size_t)n * (size_t)C, K, x, buf);
         }
         free(buf);
     }
     free(temb_all);
+}
+
+/* K Euler flow steps: x <- x + (t_{k+1} - t_k) v. */
+void oracle_head_sample(const oracle_head_params* P, const uint16_t* cond, const float* noise,
+                        const float* t_sched, int32_t K, const int32_t* idx, int32_t count,
+                        double* out) {
+    double* coef = (double*)malloc(sizeof(double) * 3 * (size_t)(K > 0 ? K : 1));
+    for (int32_t k = 0; k < K; ++k) {
+        coef[3 * k] = 1.0;
+        coef[3 * k + 1] = (double)t_sched[k + 1] - (double)t_sched[k];
+        coef[3 * k + 2] = 0.0;
+    }
+    head_sample_coef(P, cond, noise, t_sched, K, coef, NULL, 0, idx, count, out);
+    free(coef);
+}
+
+/*
+ * Other samplers on the same head (the paper's heads are also run as eps-prediction DDPM heads,
+ * "x_t = sqrt(abar_t) x + sqrt(1 - abar_t) eps", and as x_0-prediction consistency students,
+ * "x_0 = Diff_theta(x_t | t, z)"): every such step is linear in (x, head output, fresh noise), so
+ * the caller passes the three coefficients per step. t_sched [K] are the times fed to the head;
+ * coef [3K] float32 (widened); step_noise [K][n][C] float32 or NULL.
+ */
+void oracle_head_sample_coef(const oracle_head_params* P, const uint16_t* cond, const float* noise,
+                             const float* t_sched, int32_t K, const float* coef, const float* step_noise,
+                             int64_t n, const int32_t* idx, int32_t count, double* out) {
+    double* c = (double*)malloc(sizeof(double) * 3 * (size_t)(K > 0 ? K : 1));
+    for (int32_t i = 0; i < 3 * K; ++i) c[i] = (double)coef[i];
+    head_sample_coef(P, cond, noise, t_sched, K, c, step_noise, n, idx, count, out);
+    free(c);
 }
 
 /* exposed for the tests that pin the pieces separately */
