@@ -68,6 +68,41 @@ int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, float tau, ui
                            int32_t* idx, int32_t* count, float* entropy, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Block-prefix gate: the early stop as the paper's Algorithm 1, Step 1 writes it ("if H^s <
+ * tau_ent: draft_tokens <- draft_tokens[1 : i-1]; break"). Tokens come in draft blocks of
+ * `gamma` consecutive tokens (the last block may be shorter). Token i owns the
+ * rows_per_token consecutive rows i*rows_per_token .. of feat, and its indicator is the mean
+ * of their row entropies (H^s = -L_entropy: the entropy-loss equation averages over the R
+ * rows, the supplementary form over rows and heads). Scanning a block in order, the first
+ * token with indicator < tau (or NaN) drops itself and every later token of the block.
+ *
+ *   feat           dev bf16 [n * rows_per_token][d], alignment as for ardiff_entropy_gate
+ *   row_entropy    dev float [n * rows_per_token]  out (also the kernels' scratch), required
+ *   token_entropy  dev float [n]  out, or NULL
+ *   mask, idx, count   as for ardiff_entropy_gate (idx ascending)
+ *   block_len      dev int32 [ceil(n / gamma)]  out, or NULL: tokens kept in each block
+ * gamma == 1 and rows_per_token == 1 give exactly ardiff_entropy_gate's results.
+ * Allocates the same per-device scratch as ardiff_entropy_gate on first use.
+ * ------------------------------------------------------------------------------------- */
+int ardiff_entropy_gate_blocks(const void* feat, int64_t n, int32_t rows_per_token, int32_t d,
+                               int32_t gamma, float tau, float* row_entropy, float* token_entropy,
+                               uint8_t* mask, int32_t* idx, int32_t* count, int32_t* block_len,
+                               void* stream);
+
+/* Threshold from entropy statistics (the tau equation of "Entropy-Based Early Stopping in Inference
+ * Phase"): out3 = { mean(H), std(H), 0.3 * mean - 0.1 * std }, std with divisor n, all in fp64
+ * with a fixed summation order (results are reproducible run to run).
+ *   entropy dev float [n], n >= 1;  out3 dev double [3]. One CTA: meant for calibration, not the hot path. */
+int ardiff_tau_calibrate(const float* entropy, int64_t n, double* out3, void* stream);
+
+/* Accepted draft length per block (Algorithm 1, Step 4):
+ * accepted[b] = min({ i-1 : r_i > ratio_i } U { len_b }), i counted from 1 inside block b.
+ *   r, ratio  dev float [n] (the uniform draws and the density ratios p_i/q_i, both supplied by
+ *   the caller);  accepted dev int32 [ceil(n / gamma)]. */
+int ardiff_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma, int32_t* accepted,
+                         void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * Entropy gate for callers that cannot allocate device memory. (The paper has no counterpart:
  * this is a packaging variant of ardiff_entropy_gate, same operation, same results.)
  *

@@ -130,6 +130,70 @@ def ardiff_entropy_gate(feat, tau: float, mask=None, idx=None, count=None, entro
     return mask, idx, count, entropy
 
 
+def _fn(name, argtypes):
+    """A library function with its ctypes signature set (lazily, once)."""
+    fn = getattr(lib(), name)
+    if fn.argtypes is None:
+        fn.restype = ctypes.c_int
+        fn.argtypes = argtypes
+    return fn
+
+
+def ardiff_entropy_gate_blocks(feat, rows_per_token: int, gamma: int, tau: float, want_token_entropy: bool = False,
+                               stream=None):
+    """Block-prefix gate (early stop inside draft blocks of `gamma` tokens, each token owning
+    `rows_per_token` rows of feat). Returns (mask u8 [n], idx i32 [n], count i32 [1], block_len i32
+    [ceil(n/gamma)], row_entropy f32 [n*rows_per_token], token_entropy f32 [n] or None)."""
+    import torch
+    assert feat.is_cuda and feat.dtype == torch.bfloat16 and feat.dim() == 2 and feat.is_contiguous()
+    rows, d = feat.shape
+    assert rows % rows_per_token == 0
+    n = rows // rows_per_token
+    dev = feat.device
+    vp = ctypes.c_void_p
+    fn = _fn("ardiff_entropy_gate_blocks", [vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                            ctypes.c_float, vp, vp, vp, vp, vp, vp, vp])
+    mask = torch.empty((n,), dtype=torch.uint8, device=dev)
+    idx = torch.empty((max(n, 1),), dtype=torch.int32, device=dev)
+    count = torch.empty((1,), dtype=torch.int32, device=dev)
+    block_len = torch.empty((max((n + gamma - 1) // gamma, 1),), dtype=torch.int32, device=dev)
+    row_ent = torch.empty((max(rows, 1),), dtype=torch.float32, device=dev)
+    tok_ent = torch.empty((max(n, 1),), dtype=torch.float32, device=dev) if want_token_entropy else None
+    with torch.cuda.device(dev):
+        rc = fn(feat.data_ptr(), n, rows_per_token, d, gamma, float(tau), row_ent.data_ptr(),
+                tok_ent.data_ptr() if tok_ent is not None else None, mask.data_ptr(), idx.data_ptr(),
+                count.data_ptr(), block_len.data_ptr(), _stream_ptr(stream))
+    _check(rc, "ardiff_entropy_gate_blocks")
+    return mask, idx, count, block_len, row_ent, tok_ent
+
+
+def ardiff_tau_calibrate(entropy, stream=None):
+    """(mean, std, tau = 0.3 mean - 0.1 std) of a float32 CUDA tensor of entropies, as a float64 CUDA tensor [3]."""
+    import torch
+    assert entropy.is_cuda and entropy.dtype == torch.float32 and entropy.is_contiguous()
+    out = torch.empty((3,), dtype=torch.float64, device=entropy.device)
+    vp = ctypes.c_void_p
+    fn = _fn("ardiff_tau_calibrate", [vp, ctypes.c_int64, vp, vp])
+    with torch.cuda.device(entropy.device):
+        rc = fn(entropy.data_ptr(), entropy.numel(), out.data_ptr(), _stream_ptr(stream))
+    _check(rc, "ardiff_tau_calibrate")
+    return out
+
+
+def ardiff_accept_prefix(r, ratio, gamma: int, stream=None):
+    """Accepted draft length per block of `gamma`: first position with r > ratio, else the block length."""
+    import torch
+    assert r.is_cuda and r.dtype == torch.float32 and ratio.dtype == torch.float32 and r.shape == ratio.shape
+    n = r.numel()
+    out = torch.empty((max((n + gamma - 1) // gamma, 1),), dtype=torch.int32, device=r.device)
+    vp = ctypes.c_void_p
+    fn = _fn("ardiff_accept_prefix", [vp, vp, ctypes.c_int64, ctypes.c_int32, vp, vp])
+    with torch.cuda.device(r.device):
+        rc = fn(r.data_ptr(), ratio.data_ptr(), n, gamma, out.data_ptr(), _stream_ptr(stream))
+    _check(rc, "ardiff_accept_prefix")
+    return out[:(n + gamma - 1) // gamma]
+
+
 GATE_NOALLOC_MAX_BLOCKS = 1024
 GATE_NOALLOC_MAX_TOKENS = 1 << 24
 

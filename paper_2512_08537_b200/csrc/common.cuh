@@ -13,4 +13,10 @@ int gate_launch(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask
                 int32_t* count, float* entropy, int32_t* block_counts, int max_blocks, int n_sm,
                 cudaStream_t st);
 
+int entropy_rows_launch(const void* feat, int64_t rows, int32_t d, float* entropy, int n_sm, cudaStream_t st);
+int compact_launch(const uint8_t* mask, int64_t n, const int32_t* block_counts, int64_t tokens_per_block, int grid,
+                   int32_t* idx, int32_t* count, cudaStream_t st);
+int gate_scratch_get(int32_t** counts, int* max_blocks, int* sms);
+int write_zero_count(int32_t* count, cudaStream_t st);
+
 }  // namespace ardiff

@@ -153,7 +153,7 @@ gate_rows_kernel(const uint4* __restrict__ feat, int64_t n, int32_t nchunks, flo
         }
         const bool keep = (H >= tau);  // false for NaN
         if (lane == 0) {
-            mask[tok] = keep ? 1 : 0;
+            if (mask) mask[tok] = keep ? 1 : 0;
             if (entropy) entropy[tok] = H;
         }
         kept += keep ? 1 : 0;
@@ -166,7 +166,7 @@ gate_rows_kernel(const uint4* __restrict__ feat, int64_t n, int32_t nchunks, flo
         int tot = 0;
 #pragma unroll
         for (int w = 0; w < kGateWarps; ++w) tot += s_cnt[w];
-        block_counts[blockIdx.x] = tot;
+        if (block_counts) block_counts[blockIdx.x] = tot;
     }
 }
 
@@ -205,7 +205,7 @@ gate_rows_generic_kernel(const uint16_t* __restrict__ feat, int64_t n, int32_t d
         const float H = logf(S) - kLn2 * (T / S);
         const bool keep = (H >= tau);
         if (lane == 0) {
-            mask[tok] = keep ? 1 : 0;
+            if (mask) mask[tok] = keep ? 1 : 0;
             if (entropy) entropy[tok] = H;
         }
         kept += keep ? 1 : 0;
@@ -216,7 +216,7 @@ gate_rows_generic_kernel(const uint16_t* __restrict__ feat, int64_t n, int32_t d
     if (threadIdx.x == 0) {
         int tot = 0;
         for (int w = 0; w < kGateWarps; ++w) tot += s_cnt[w];
-        block_counts[blockIdx.x] = tot;
+        if (block_counts) block_counts[blockIdx.x] = tot;
     }
 }
 
@@ -346,6 +346,54 @@ int gate_launch(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask
     }
     compact_kernel<<<grid, kGateThreads, 0, st>>>(mask, n, block_counts, tpb, idx, count);
     set_launch_count(2);
+    return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+}
+
+// Row entropies only (no threshold, no compaction): entropy[i] = H of row i.
+int entropy_rows_launch(const void* feat, int64_t rows, int32_t d, float* entropy, int n_sm, cudaStream_t st) {
+    if (rows < 0 || rows >= (int64_t)1 << 31 || d < 1 || d > 65536) return ARDIFF_ERR_SHAPE;
+    if (rows == 0) return ARDIFF_OK;
+    if (!feat || !entropy) return ARDIFF_ERR_NULL;
+    const bool vec = (d % 8 == 0) && (d <= 8192);
+    if (vec && (reinterpret_cast<uintptr_t>(feat) & 15u)) return ARDIFF_ERR_ALIGN;
+    if (!vec && (reinterpret_cast<uintptr_t>(feat) & 1u)) return ARDIFF_ERR_ALIGN;
+    int64_t want = (int64_t)n_sm * 8;
+    int64_t tpb = (rows + want - 1) / want;
+    if (tpb < kGateWarps) tpb = kGateWarps;
+    const int grid = (int)((rows + tpb - 1) / tpb);
+    const float tau = 0.f;
+    if (vec) {
+        const int need = (d / 8 + 31) / 32;
+        if (need <= 1) launch_rows<1>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 2) launch_rows<2>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 4) launch_rows<4>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 8) launch_rows<8>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 12) launch_rows<12>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 16) launch_rows<16>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 20) launch_rows<20>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else if (need <= 24) launch_rows<24>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+        else launch_rows<32>(grid, st, feat, rows, d, tau, nullptr, entropy, nullptr, tpb);
+    } else {
+        gate_rows_generic_kernel<<<grid, kGateThreads, 0, st>>>(reinterpret_cast<const uint16_t*>(feat), rows, d, tau,
+                                                               nullptr, entropy, nullptr, tpb);
+    }
+    return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+}
+
+// Stable compaction of a mask whose per-block kept counts (blocks of tokens_per_block tokens) are known.
+int compact_launch(const uint8_t* mask, int64_t n, const int32_t* block_counts, int64_t tokens_per_block, int grid,
+                   int32_t* idx, int32_t* count, cudaStream_t st) {
+    compact_kernel<<<grid, kGateThreads, 0, st>>>(mask, n, block_counts, tokens_per_block, idx, count);
+    return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+}
+
+int gate_scratch_get(int32_t** counts, int* max_blocks, int* sms) {
+    *max_blocks = kMaxGateBlocks;
+    return gate_scratch(counts, sms);
+}
+
+int write_zero_count(int32_t* count, cudaStream_t st) {
+    write_zero_count_kernel<<<1, 1, 0, st>>>(count);
     return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
 }
 
