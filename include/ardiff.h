@@ -210,6 +210,25 @@ int ardiff_head_sample(const ardiff_head* head, const void* cond, const float* n
                        const float* t_sched, int32_t K, const int32_t* idx, const int32_t* count,
                        float* out, void* stream);
 
+/*
+ * The same head under another sampler. The paper's heads are also run as eps-prediction DDPM
+ * heads ("x_t = sqrt(abar_t) x + sqrt(1 - abar_t) eps", AR+Diffusion Hybrid Paradigm) and, after
+ * consistency distillation, as x_0-predicting students ("x_0 = Diff_theta(x_t | t, z)"); every such
+ * sampler step is linear in the state, the head output v and fresh noise, so the caller passes
+ * three coefficients per step:  x <- ax_k x + av_k v + an_k z_k.
+ *   t_in        HOST float [K]: the time fed to the head at step k
+ *   coef        HOST float [3K]: ax_0, av_0, an_0, ax_1, ...   (Euler flow: 1, t_{k+1} - t_k, 0;
+ *               deterministic eps-prediction step from abar to abar': ax = sqrt(abar'/abar),
+ *               av = sqrt(1 - abar') - ax sqrt(1 - abar), an = 0; x_0-prediction with re-noising:
+ *               ax = 0, av = sqrt(abar'), an = sqrt(1 - abar'))
+ *   step_noise  dev float [K][n][C], 16-byte aligned, or NULL (then an_k is ignored); row i of
+ *               slice k is the fresh noise of token i at step k;  n = rows of noise / out
+ * Everything else as ardiff_head_sample (which is this call with the Euler coefficients).
+ */
+int ardiff_head_sample_coef(const ardiff_head* head, const void* cond, const float* noise,
+                            const float* t_in, int32_t K, const float* coef, const float* step_noise,
+                            int64_t n, const int32_t* idx, const int32_t* count, float* out, void* stream);
+
 /* Waits for `stream`, then returns the head's device status word: ARDIFF_OK, or
  * ARDIFF_ERR_TIMEOUT if any bounded wait of an earlier sample call ran out, or
  * ARDIFF_ERR_SHAPE if *count exceeded max_tokens. Clears it. */

@@ -256,6 +256,31 @@ class Head:
         _check(rc, "ardiff_head_sample")
         return out
 
+    def ardiff_head_sample_coef(self, cond, noise, t_in, coef, idx, count, out, step_noise=None, stream=None):
+        """K = len(t_in) head evaluations, each followed by x <- ax x + av v + an z_k.
+        coef: [K, 3] (ax, av, an); step_noise: float32 CUDA tensor [K, n, C] or None."""
+        import numpy as np
+        import torch
+        assert cond.is_cuda and cond.dtype == torch.bfloat16 and cond.is_contiguous()
+        assert noise.is_cuda and noise.dtype == torch.float32 and noise.is_contiguous()
+        assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+        ts = np.ascontiguousarray(t_in, dtype=np.float32)
+        cf = np.ascontiguousarray(coef, dtype=np.float32)
+        K = ts.shape[0]
+        assert cf.shape == (K, 3)
+        n = noise.shape[0]
+        if step_noise is not None:
+            assert step_noise.is_cuda and step_noise.dtype == torch.float32 and step_noise.is_contiguous()
+            assert tuple(step_noise.shape) == (K, n, noise.shape[1])
+        vp = ctypes.c_void_p
+        fn = _fn("ardiff_head_sample_coef", [vp, vp, vp, vp, ctypes.c_int32, vp, vp, ctypes.c_int64, vp, vp, vp, vp])
+        with torch.cuda.device(cond.device):
+            rc = fn(self._h, cond.data_ptr(), noise.data_ptr(), ts.ctypes.data, K, cf.ctypes.data,
+                    step_noise.data_ptr() if step_noise is not None else None, n, idx.data_ptr(), count.data_ptr(),
+                    out.data_ptr(), _stream_ptr(stream))
+        _check(rc, "ardiff_head_sample_coef")
+        return out
+
     def status(self, stream=None) -> int:
         return int(lib().ardiff_head_status(self._h, _stream_ptr(stream)))
 

@@ -119,7 +119,9 @@ struct HeadParams {
     int* status;
     int* abort_flag;
     long long* trace;
-    float dt[KMAX];
+    const float* step_noise;                // [K][n][C] fresh noise of the sampler steps, or nullptr
+    long long step_stride;                  // n * C
+    float ax[KMAX], av[KMAX], an[KMAX];     // sampler step k: x <- ax x + av v + an z_k
 };
 
 struct Packed { uint32_t w0, w1, w2, w3, w4; };
@@ -471,16 +473,21 @@ __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, u
     }
 }
 
-// v = acc + bout ; x += dt_k v ; bf16 copy for the next in-projection ; last step: out[idx[j]] = x
+// v = acc + bout ; x <- ax_k x + av_k v + an_k z_k ; bf16 copy for the next in-projection ; last step: out[idx[j]] = x
 __device__ __forceinline__ void epi_out(const HeadParams& P, const Item& it, uint32_t tacc, int grow,
                                         int j, int count) {
-    const float dt = P.dt[it.k];
+    const float ax = P.ax[it.k], av = P.av[it.k], an = P.an[it.k];
     float* xrow = P.x + (size_t)grow * P.C;
     bf16* xbrow = P.xb + (size_t)grow * XB_COLS;
     const float* bias = P.bias_cat + it.b_row;
     const bool last = (it.k == P.K - 1);
     float* orow = nullptr;
-    if (last && j < count) orow = P.out + (size_t)__ldg(P.idx + j) * P.C;
+    const float* zrow = nullptr;
+    if (j < count && (last || P.step_noise)) {
+        const size_t tok = (size_t)__ldg(P.idx + j);
+        if (last) orow = P.out + tok * P.C;
+        if (P.step_noise) zrow = P.step_noise + (size_t)it.k * (size_t)P.step_stride + tok * P.C;
+    }
     for (int cc = 0; cc < P.C / 16; ++cc) {
         uint32_t r[16];
         ptx::tmem_ld_32x32b_x16(tacc + cc * 16, r);
@@ -490,10 +497,16 @@ __device__ __forceinline__ void epi_out(const HeadParams& P, const Item& it, uin
         for (int i = 0; i < 16; i += 4) {
             const float4 b = __ldg(reinterpret_cast<const float4*>(bias + cc * 16 + i));
             const float4 xo = ptx::ldcg_f4(xrow + cc * 16 + i);
-            xn[i] = fmaf(dt, __uint_as_float(r[i]) + b.x, xo.x);
-            xn[i + 1] = fmaf(dt, __uint_as_float(r[i + 1]) + b.y, xo.y);
-            xn[i + 2] = fmaf(dt, __uint_as_float(r[i + 2]) + b.z, xo.z);
-            xn[i + 3] = fmaf(dt, __uint_as_float(r[i + 3]) + b.w, xo.w);
+            float4 base = make_float4(ax * xo.x, ax * xo.y, ax * xo.z, ax * xo.w);   // ax = 1: exactly x
+            if (zrow) {
+                const float4 z = __ldg(reinterpret_cast<const float4*>(zrow + cc * 16 + i));
+                base.x = fmaf(an, z.x, base.x); base.y = fmaf(an, z.y, base.y);
+                base.z = fmaf(an, z.z, base.z); base.w = fmaf(an, z.w, base.w);
+            }
+            xn[i] = fmaf(av, __uint_as_float(r[i]) + b.x, base.x);
+            xn[i + 1] = fmaf(av, __uint_as_float(r[i + 1]) + b.y, base.y);
+            xn[i + 2] = fmaf(av, __uint_as_float(r[i + 2]) + b.z, base.z);
+            xn[i + 3] = fmaf(av, __uint_as_float(r[i + 3]) + b.w, base.w);
         }
 #pragma unroll
         for (int i = 0; i < 16; i += 4) {
@@ -1284,12 +1297,15 @@ extern "C" int ardiff_head_destroy(ardiff_head* H) {
     return ARDIFF_OK;
 }
 
-extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const float* noise,
-                                  const float* t_sched, int32_t K, const int32_t* idx, const int32_t* count,
-                                  float* out, void* stream) {
+namespace {
+// t_in [K]: the times fed to the head; coef [3K]: (ax, av, an) of every step
+int head_sample_impl(const ardiff_head* H, const void* cond, const float* noise, const float* t_sched, int32_t K,
+                     const float* coef, const float* step_noise, int64_t n_rows, const int32_t* idx,
+                     const int32_t* count, float* out, void* stream) {
     if (!H || !idx || !count) return ARDIFF_ERR_NULL;
     if (K < 0 || K > H->d.K_max) return ARDIFF_ERR_SHAPE;
-    if (H->d.max_tokens > 0 && (!cond || !noise || !out || !t_sched)) return ARDIFF_ERR_NULL;
+    if (H->d.max_tokens > 0 && (!cond || !noise || !out || !t_sched || !coef)) return ARDIFF_ERR_NULL;
+    if (step_noise && (n_rows < 1 || (reinterpret_cast<uintptr_t>(step_noise) & 15u))) return ARDIFF_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(cond) & 15u) return ARDIFF_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(noise) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u))
         return ARDIFF_ERR_ALIGN;
@@ -1329,7 +1345,11 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
     P.bias_cat = H->bias_cat; P.bc = H->bc; P.bin = H->bin; P.temb = H->temb;
     P.counters = H->counters; P.status = H->status; P.abort_flag = H->status + 1;
     P.trace = H->trace;
-    for (int k = 0; k < K; ++k) P.dt[k] = (float)((double)t_sched[k + 1] - (double)t_sched[k]);
+    for (int k = 0; k < K; ++k) {
+        P.ax[k] = coef[3 * k]; P.av[k] = coef[3 * k + 1]; P.an[k] = coef[3 * k + 2];
+    }
+    P.step_noise = step_noise;
+    P.step_stride = (long long)n_rows * C;
 
     ardiff_head* Hm = const_cast<ardiff_head*>(H);
     if (H->timing) cudaEventRecord(H->ev0, st);
@@ -1361,6 +1381,28 @@ extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const 
     launches += 1;
     ardiff::set_launch_count(launches);
     return ARDIFF_OK;
+}
+}  // namespace
+
+extern "C" int ardiff_head_sample(const ardiff_head* H, const void* cond, const float* noise,
+                                  const float* t_sched, int32_t K, const int32_t* idx, const int32_t* count,
+                                  float* out, void* stream) {
+    if (K < 0 || K > KMAX) return ARDIFF_ERR_SHAPE;
+    if (K > 0 && !t_sched) return ARDIFF_ERR_NULL;
+    float coef[3 * KMAX + 3];
+    for (int k = 0; k < K; ++k) {      // Euler flow step: x <- x + (t_{k+1} - t_k) v
+        coef[3 * k] = 1.0f;
+        coef[3 * k + 1] = (float)((double)t_sched[k + 1] - (double)t_sched[k]);
+        coef[3 * k + 2] = 0.0f;
+    }
+    return head_sample_impl(H, cond, noise, t_sched, K, coef, nullptr, 0, idx, count, out, stream);
+}
+
+extern "C" int ardiff_head_sample_coef(const ardiff_head* H, const void* cond, const float* noise,
+                                       const float* t_in, int32_t K, const float* coef, const float* step_noise,
+                                       int64_t n, const int32_t* idx, const int32_t* count, float* out,
+                                       void* stream) {
+    return head_sample_impl(H, cond, noise, t_in, K, coef, step_noise, n, idx, count, out, stream);
 }
 
 extern "C" int ardiff_head_set_timing(ardiff_head* H, int on) {

@@ -163,3 +163,31 @@ def test_full_size_gate_stress_sampled_rows_and_properties():
         want_idx = torch.nonzero(mask, as_tuple=False).flatten().to(torch.int32)
         assert torch.equal(idx[:c], want_idx)
         assert abs(c / wl.n - (1 - q)) < 0.03
+    # the survivors of the last (99 % filtered) pass feed the cfg2-shaped head: under-filled grid, ragged tail
+    S = c
+    idx_h = idx[:S].cpu().numpy()
+    w, t = synth.head_weights(wl), synth.t_sched(wl.K)
+    cond = torch.empty((wl.n, wl.Dc), dtype=torch.bfloat16, device=dev)
+    noise = torch.empty((wl.n, wl.C), dtype=torch.float32, device=dev)
+    big = 1 << 17
+    for r0 in range(0, wl.n, big):
+        cond[r0:r0 + big] = dev_bf16(synth.cond(wl, r0, big))
+        noise[r0:r0 + big] = torch.from_numpy(synth.noise(wl, r0, big)).to(dev)
+    head = ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K, wl.n, w)
+    out = torch.full((wl.n, wl.C), -777.0, dtype=torch.float32, device=dev)
+    head.ardiff_head_sample(cond, noise, t, idx, count, out)
+    assert head.status() == 0
+    pos = np.unique(np.concatenate([np.arange(0, 12), np.arange(S - (S % 128 or 128), S)[-12:],
+                                    rng.integers(0, S, size=24)]))
+    toks = idx_h[pos]
+    small = synth.workload("cfg5", n=len(toks))
+    cond_s = np.concatenate([synth.cond(wl, int(tk), 1) for tk in toks])
+    noise_s = np.concatenate([synth.noise(wl, int(tk), 1) for tk in toks])
+    want = oracle.head_sample(w, cond_s, noise_s, t, np.arange(len(toks), dtype=np.int32))
+    got = out[torch.from_numpy(toks.astype(np.int64)).to(dev)].cpu().numpy().astype(np.float64)
+    err = np.abs(got - want).max(axis=1) / np.sqrt((want ** 2).mean(axis=1))
+    assert err.max() <= 2e-2, err.max()
+    written = (out[:, 0] != -777.0)
+    assert int(written.sum().item()) == S and bool(written[torch.from_numpy(idx_h.astype(np.int64)).to(dev)].all())
+    assert bool(torch.isfinite(out[written]).all())
+    head.close()

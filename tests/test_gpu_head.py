@@ -202,3 +202,54 @@ def test_bad_arguments_are_rejected():
     assert lib.ardiff_head_sample(head._h, p, p, t.ctypes.data, 4, None, p, p, None) == ardiff.ARDIFF_ERR_NULL
     assert lib.ardiff_head_sample(head._h, p + 2, p, t.ctypes.data, 4, p, p, p, None) == ardiff.ARDIFF_ERR_ALIGN
     head.close()
+
+
+def ddim_coef(abar):
+    """Deterministic eps-prediction steps along abar[0] -> abar[1] -> ... (coefficients of x and eps)."""
+    abar = np.asarray(abar, np.float64)
+    ax = np.sqrt(abar[1:] / abar[:-1])
+    av = np.sqrt(1 - abar[1:]) - ax * np.sqrt(1 - abar[:-1])
+    return np.stack([ax, av, np.zeros_like(ax)], axis=1).astype(np.float32)
+
+
+@pytest.mark.parametrize("sampler", ["euler", "ddim", "x0_renoise"])
+def test_linear_sampler_steps(sampler):
+    """Other samplers on the same head: every step is x <- ax x + av v + an z_k."""
+    dev = require_cuda()
+    wl = synth.workload("cfg1", n=300, K=4)
+    # Euler and eps-prediction keep the state (ax != 0) and run on the harder 1/sqrt(fan_in) weights; the
+    # x0-prediction sampler returns the head's raw last output after two compounding passes and runs on
+    # the workloads' own weight recipe, N(0, 0.02)
+    w = synth.head_weights(wl, std=0.02 if sampler == "x0_renoise" else None)
+    cond_bits, noise = synth.cond(wl), synth.noise(wl)
+    idx_np = np.random.default_rng(7).permutation(wl.n)[:211].astype(np.int32)
+    z = None
+    if sampler == "euler":
+        t = np.array([0.0, 0.2, 0.5, 0.9, 1.0], np.float32)
+        t_in = t[:-1]
+        coef = np.stack([np.ones(4), t[1:].astype(np.float64) - t[:-1].astype(np.float64), np.zeros(4)], 1).astype(np.float32)
+    elif sampler == "ddim":
+        t_in = np.array([0.95, 0.7, 0.45, 0.2], np.float32)
+        coef = ddim_coef([0.05, 0.3, 0.6, 0.85, 0.999])
+    else:
+        # two-step consistency sampling: predict x0, re-noise to abar = 0.5, predict x0 again. The output
+        # is the head's last raw prediction (ax = 0 discards the state), so nothing props up its RMS.
+        t_in = np.array([0.95, 0.5], np.float32)
+        abn = np.array([0.5, 1.0])
+        coef = np.stack([np.zeros(2), np.sqrt(abn), np.sqrt(1 - abn)], 1).astype(np.float32)
+        z = np.random.default_rng(8).standard_normal((2, wl.n, wl.C)).astype(np.float32)
+    want = oracle.head_sample_coef(w, cond_bits, noise, t_in, coef, idx_np, step_noise=z)
+    head = make_head(wl, w)
+    idx = torch.from_numpy(idx_np).to(dev)
+    count = torch.tensor([len(idx_np)], dtype=torch.int32, device=dev)
+    out = torch.full(noise.shape, SENTINEL, dtype=torch.float32, device=dev)
+    head.ardiff_head_sample_coef(dev_bf16(cond_bits), dev_f32(noise), t_in, coef, idx, count, out,
+                                 step_noise=None if z is None else torch.from_numpy(z).to(dev))
+    assert head.status() == 0
+    got = out.cpu().numpy()
+    assert_parity(got, want, idx_np, sampler)
+    assert np.all(got[np.setdiff1d(np.arange(wl.n), idx_np)] == SENTINEL)
+    if sampler == "euler":                 # the Euler entry point is this call with the Euler coefficients
+        got2 = run_head(head, cond_bits, noise, np.array([0.0, 0.2, 0.5, 0.9, 1.0], np.float32), idx_np)
+        assert np.array_equal(got2[idx_np], got[idx_np])
+    head.close()
