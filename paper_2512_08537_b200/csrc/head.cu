@@ -621,12 +621,21 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         uint32_t seq = 0;
         bool aborted = false;
         ItemStream ist;
-        Item it;
+        Item it, nx;
         TRACE_DECL
-        while (ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, it)) {
-            if (it.type == OP_GATHER) continue;
+        // next item with operands to load (gather items have none)
+        auto next_item = [&](Item& dst) {
+            bool have;
+            do have = ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, dst);
+            while (have && dst.type == OP_GATHER);
+            return have;
+        };
+        bool have = next_item(it);
+        bool pre_ok = false;    // the dependencies of `it` were already seen complete while the item before it streamed
+        while (have) {
+            const bool have_nx = next_item(nx);
             bool ok = true;
-            if (lane == 0) {
+            if (lane == 0 && !pre_ok) {
                 const int* ctr = P.counters + (size_t)it.abs_m * CTRS;
                 ok = wait_counters(ctr, it.needA, it.needB ? ctr + it.gsel : nullptr, it.needB, P);
             }
@@ -640,6 +649,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             const void* map_b = P.maps + it.map_b;
             const int b_rows = it.umma_n / 2;                         // rows of B this CTA stages
             const uint32_t tx = 2u * (A_BYTES + (uint32_t)b_rows * BK * 2);
+            const int peek_kb = it.kblocks > 3 ? it.kblocks - 3 : 0;
+            int pv1 = 0, pv2 = 0;      // the next item's counters, read while this item still streams
             for (int kb = 0; kb < it.kblocks; ++kb) {
                 ok = wait_mbar(empty_bar(stage), phase ^ 1u, P);
                 ok = __all_sync(0xffffffffu, ok);
@@ -651,6 +662,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                     if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
                     ptx::tma_load_2d_pair(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
                     ptx::tma_load_2d_pair(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row + rank * b_rows);
+                    if (kb == peek_kb && have_nx) {
+                        // issued here, looked at only after the last slice went out
+                        const int* ctr = P.counters + (size_t)nx.abs_m * CTRS;
+                        pv1 = ptx::ld_acquire_gpu(ctr);
+                        pv2 = nx.needB ? ptx::ld_acquire_gpu(ctr + nx.gsel) : 0;
+                    }
                 }
                 issued |= 1u << stage;
                 issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
@@ -658,6 +675,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             }
             TRACE(0, 2); TRACE_TYPE(0); TRACE_NEXT();
             if (!ok) { aborted = true; break; }
+            const int pre = (have_nx && pv1 >= nx.needA && pv2 >= nx.needB) ? 1 : 0;
+            pre_ok = __shfl_sync(0xffffffffu, pre, 0) != 0;
+            it = nx;
+            have = have_nx;
         }
         // own copies in flight must have landed before the CTA exits. In the even CTA the full
         // barriers are local: wait for every stage's last issue. The odd CTA's loads are counted on
@@ -752,9 +773,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 ++seq;
                 if (!ok) break;
                 if (ew == 0) TRACE(2, 0);
-                ptx::fence_proxy_async();
                 const EpiIO io = epi_io(it, half);
                 const bool has_loads = (io.ldF >= 0) || (io.ldH >= 0);
+                if (has_loads) ptx::fence_proxy_async();   // other CTAs' writes -> this warp's TMA reads
                 const int row0 = it.slot_row0 + quarter * 32;
                 auto issue_load = [&](int j) {
                     const int b = j & 1;
@@ -827,8 +848,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             }
             if (fail) break;
             // publish: this warp's global writes, then one tick of the token tile's counter
-            __threadfence();
-            ptx::fence_proxy_async();
+            // The release below is cumulative: it covers this lane's completed TMA stores and, through the
+            // warp barrier, the other lanes' plain stores. Rows written with plain stores that other CTAs
+            // read by TMA (z, xb) additionally need the generic -> async proxy fence on the writer's side.
+            if (it.type == OP_GATHER || it.type == OP_OUT) ptx::fence_proxy_async();
             __syncwarp();
             if (lane == 0)
                 ptx::red_release_gpu_add(P.counters + (size_t)it.abs_m * CTRS + (it.type == OP_GATE ? it.gsel : 0), 1);
