@@ -30,7 +30,7 @@ METRIC = "gated draft tokens/sec through K-step head"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 512 << 20
 # dram bytes per launch of the head kernel from the ncu capture summarised under profiles/
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {"cfg2": 4.325e9}
 
 
 def peaks():
@@ -121,13 +121,24 @@ class ClockSampler:
             import pynvml
             pynvml.nvmlInit()
             self.nv = pynvml
-            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
-            phys = dev_index
-            if visible:
-                ids = [v.strip() for v in visible.split(",") if v.strip()]
-                if dev_index < len(ids) and ids[dev_index].isdigit():
-                    phys = int(ids[dev_index])
-            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.h = None
+            try:
+                # the NVML handle of the very GPU torch uses (CUDA_VISIBLE_DEVICES may reorder or name UUIDs)
+                import torch
+                uuid = str(torch.cuda.get_device_properties(dev_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = None
+            if self.h is None:
+                visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+                phys = dev_index
+                if visible:
+                    ids = [v.strip() for v in visible.split(",") if v.strip()]
+                    if dev_index < len(ids) and ids[dev_index].isdigit():
+                        phys = int(ids[dev_index])
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
             self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
         except Exception:
             self.nv = None
@@ -138,8 +149,9 @@ class ClockSampler:
 
     def _run(self):
         nv = self.nv
-        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
-                 "hw_thermal_slowdown": 0x40}
+        names = {"applications_clocks_setting": 0x2, "sw_power_cap": 0x4, "hw_slowdown": 0x8, "sync_boost": 0x10,
+                 "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40, "hw_power_brake_slowdown": 0x80,
+                 "display_clock_setting": 0x100}
         while not self._stop.is_set():
             try:
                 self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
