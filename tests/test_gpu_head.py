@@ -253,3 +253,21 @@ def test_linear_sampler_steps(sampler):
         got2 = run_head(head, cond_bits, noise, np.array([0.0, 0.2, 0.5, 0.9, 1.0], np.float32), idx_np)
         assert np.array_equal(got2[idx_np], got[idx_np])
     head.close()
+
+
+@pytest.mark.parametrize("shape", [dict(W=4096, L=1, K=1, C=32, Dc=64, n=130),
+                                   dict(W=2048, L=2, K=2, C=64, Dc=128, n=300),
+                                   dict(W=256, L=5, K=3, C=48, Dc=1024, n=257),
+                                   dict(W=512, L=1, K=64, C=16, Dc=64, n=40)])
+def test_extreme_shapes(shape):
+    """Widest head (16 column tiles, 32 LayerNorm partials per row), the largest token dim, an odd number
+    of blocks (gate buffers alternate by block parity), the largest step count."""
+    n = shape.pop("n")
+    wl = synth.workload("cfg1", n=n, **shape)
+    w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    idx = np.arange(n, dtype=np.int32)
+    want = oracle.head_sample(w, cond_bits, noise, t, idx)
+    head = make_head(wl, w)
+    got = run_head(head, cond_bits, noise, t, idx)
+    assert_parity(got, want, idx, str(shape))
+    head.close()
