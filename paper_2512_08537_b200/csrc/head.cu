@@ -76,10 +76,10 @@ constexpr int TRACE_ITEMS = 4096;
 #define TRACE_NEXT()
 #endif
 
-enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_SS, OP_GATE, OP_G1, OP_G2, OP_FSS, OP_OUT, OP_END = 15 };
+enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_SS, OP_GATE, OP_G1, OP_G2, OP_FSS, OP_OUT, OP_NOP, OP_END = 15 };
 enum MapId : int {
     MAP_Z = 0, MAP_XB, MAP_S, MAP_U, MAP_A, MAP_WC, MAP_WIN, MAP_WCAT, MAP_WOUT,   // GEMM operands
-    EMAP_H, EMAP_C, EMAP_S, EMAP_U, EMAP_A, EMAP_G0, EMAP_G1,                       // epilogue slabs
+    EMAP_H, EMAP_S, EMAP_U, EMAP_A, EMAP_G0, EMAP_G1,                       // epilogue slabs
     MAP_COUNT
 };
 
@@ -93,15 +93,14 @@ struct Phase {
     int cum;       // column tiles per token tile in the phases before it within one step
     int b_row0;    // first row of the layer's weights in the B matrix
     int offA;      // chain items of this step that must be complete (per token tile)
-    int gsel;      // 0: none; 1/2: gate counter (even/odd blocks) bumped (OP_GATE) or awaited (OP_G2)
-    int goff;      // OP_G2: gate items of that parity that must be complete within this step
+    int kplus;     // OP_GATE: 1 when the gate belongs to block `block` of the NEXT step
 };
 
 struct HeadParams {
     int C, Dc, W, L, K, NT, TGu, slots;     // NT = W/256, TGu = largest group in units, slots = scratch tiles
     int T_pro, T_step, T_chain;             // items per unit: prologue, one step, whole call
     int C_pro, C_step, C_total;             // chain-counter items per token tile: prologue, one step, whole call
-    int gcnt[2];                            // gate items per step and token tile with even / odd block index
+    int R;                                  // rows of the scratch arrays (slots * 128)
     int max_tokens;
     const Phase* phases;
     const uint16_t* cum2phase;              // [T_step]: phase that holds the c-th column tile of a step
@@ -112,7 +111,7 @@ struct HeadParams {
     const int* count;
     float* out;
     bf16 *z, *xb, *s, *u, *a, *g0, *g1;
-    float *x, *c, *h;
+    float *x, *h;
     float2* stats;
     const float *bias_cat, *bc, *bin, *temb;
     int* counters;
@@ -127,7 +126,7 @@ struct HeadParams {
 struct Packed { uint32_t w0, w1, w2, w3, w4; };
 
 struct Item {
-    int type, abs_m, slot_row0, nt, k, block, gsel;
+    int type, abs_m, slot_row0, a_row0, nt, k, block, gsel;   // a_row0: first row of the A operand in its tensor
     int needA, needB;
     int map_a, map_b, b_row, kblocks, umma_n;
 };
@@ -205,13 +204,21 @@ __device__ __forceinline__ Packed decode_packed(const HeadParams& P, int MTu, in
     if (r < pro) {
         if (r < mtg) {
             type = OP_GATHER; m = r;
-        } else {
+        } else if (r < mtg + mtg * P.NT) {
             r -= mtg;
             m = r / P.NT;
             nt = r - m * P.NT;
             type = OP_COND;
             needA = EPI_WARPS;            // the gather of this token tile
             b_row = nt * BN;
+        } else {
+            // the gate of step 0, block 0 (gate number 0): needs s_0, i.e. the conditioning items
+            r -= mtg + mtg * P.NT;
+            m = r / P.NT;
+            nt = r - m * P.NT;
+            type = OP_GATE; gsel = 1;
+            needA = EPI_WARPS * P.C_pro;
+            b_row = 2 * P.W + nt * BN;
         }
     } else {
         r -= pro;
@@ -223,10 +230,20 @@ __device__ __forceinline__ Packed decode_packed(const HeadParams& P, int MTu, in
         const int q = r - p.cum * mtg;
         m = q / p.ntiles;
         nt = p.tile0 + (q - m * p.ntiles);
-        type = p.type; block = p.block; gsel = p.gsel;
+        type = p.type; block = p.block;
         needA = EPI_WARPS * (P.C_pro + k * P.C_step + p.offA);
-        if (type == OP_G2) needB = EPI_WARPS * (k * P.gcnt[gsel - 1] + p.goff);
         b_row = p.b_row0 + nt * BN;
+        // gates are numbered q = step * L + block over the whole call; gate q lives in buffer q & 1 and
+        // ticks counter 1 + (q & 1), so the (q >> 1) + 1 -th gate of that parity is complete at NT * that many ticks
+        if (type == OP_GATE) {
+            k += p.kplus;                         // the step whose s it reads
+            if (k >= P.K) type = OP_NOP;          // beyond the last step: nothing to do
+            else gsel = 1 + ((k * P.L + block) & 1);
+        } else if (type == OP_G2) {
+            const int q = k * P.L + block;
+            gsel = 1 + (q & 1);
+            needB = EPI_WARPS * P.NT * ((q >> 1) + 1);
+        }
     }
     const int abs_m = (m0 + m) * 2 + rank;
     pk.w0 = (uint32_t)abs_m | ((uint32_t)type << 24);
@@ -245,7 +262,11 @@ __device__ __forceinline__ void unpack_item(const HeadParams& P, const Packed& p
     it.gsel = (int)(pk.w1 >> 24);
     it.needA = (int)pk.w2; it.needB = (int)pk.w3; it.b_row = (int)pk.w4;
     it.kblocks = P.W / BK; it.umma_n = BN; it.map_b = MAP_WCAT; it.map_a = MAP_S;
+    it.a_row0 = it.slot_row0;
     switch (it.type) {
+        case OP_SS:
+        case OP_GATE:
+        case OP_FSS: it.a_row0 = it.k * P.R + it.slot_row0; break;     // s of step k
         case OP_COND: it.map_a = MAP_Z; it.map_b = MAP_WC; it.kblocks = P.Dc / BK; break;
         case OP_IN: it.map_a = MAP_XB; it.map_b = MAP_WIN; it.kblocks = 1; break;
         case OP_G1: it.map_a = MAP_U; break;
@@ -308,8 +329,8 @@ struct EpiIO {            // what one warp moves per 32-column chunk of one item
 __device__ __forceinline__ EpiIO epi_io(const Item& it, int half) {
     EpiIO io{4, half * 128, it.nt * BN + half * 128, -1, -1, -1, -1};
     switch (it.type) {
-        case OP_COND: io.stF = EMAP_C; break;
-        case OP_IN: io.ldF = EMAP_C; io.stF = EMAP_H; io.stH = EMAP_S; break;
+        case OP_COND: break;          // own path: one bf16 slab per step
+        case OP_IN: io.stF = EMAP_H; break;
         case OP_SS:
         case OP_FSS:
             io.nch = 2; io.acc0 = half * 64; io.col0 = it.nt * 128 + half * 64;
@@ -407,25 +428,13 @@ __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, u
                                           float rstd) {
     float v[32];
     switch (it.type) {
-        case OP_COND: {                       // c = acc + bc
-            load_acc32(acc, v);
-            add_bias32(v, P.bc + col);
-            slabF_write(bufF, r, v);
-            break;
-        }
-        case OP_IN: {                         // h = acc + bin ; s = SiLU(c + temb_k)
+        case OP_IN: {                         // h = acc + bin
             load_acc32(acc, v);
             add_bias32(v, P.bin + col);
             if (first) st.init(v[0]);
 #pragma unroll
             for (int i = 0; i < 32; ++i) st.add(v[i]);
-            float cv[32];
-            slabF_read(bufF, r, cv);
             slabF_write(bufF, r, v);
-            add_bias32(cv, P.temb + (size_t)it.k * P.W + col);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) cv[i] = silu_f(cv[i]);
-            slabH_write(bufH, r, cv);
             break;
         }
         case OP_SS:
@@ -627,7 +636,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         auto next_item = [&](Item& dst) {
             bool have;
             do have = ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, dst);
-            while (have && dst.type == OP_GATHER);
+            while (have && (dst.type == OP_GATHER || dst.type == OP_NOP));
             return have;
         };
         bool have = next_item(it);
@@ -660,7 +669,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                     const uint32_t sa = smem_base + stage * STAGE_BYTES;
                     // the even CTA arms its barrier for the bytes of both CTAs
                     if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-                    ptx::tma_load_2d_pair(sa, map_a, full_bar(stage), kb * BK, it.slot_row0);
+                    ptx::tma_load_2d_pair(sa, map_a, full_bar(stage), kb * BK, it.a_row0);
                     ptx::tma_load_2d_pair(sa + A_BYTES, map_b, full_bar(stage), kb * BK, it.b_row + rank * b_rows);
                     if (kb == peek_kb && have_nx) {
                         // issued here, looked at only after the last slice went out
@@ -701,7 +710,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             Item it;
             TRACE_DECL
             while (ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, it)) {
-                if (it.type == OP_GATHER) continue;
+                if (it.type == OP_GATHER || it.type == OP_NOP) continue;
                 const uint32_t buf = acc_iter & 1u;
                 const uint32_t acc_phase = (acc_iter >> 1) & 1u;
                 bool ok = wait_mbar(tempty_bar(buf), acc_phase ^ 1u, P);
@@ -757,6 +766,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         TRACE_DECL
         while (ist.next(P, MTu, tgu, rank, unit_id, n_units, total, lane, it)) {
             bool fail = false;
+            if (it.type == OP_NOP) continue;
             if (it.type == OP_GATHER) {
                 bool ok = true;
                 // the scratch slot is free once the token tile that used it before has run its whole chain
@@ -802,6 +812,41 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 const uint32_t tacc = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
                 if (it.type == OP_OUT) {
                     if (!fail && half == 0) epi_out(P, it, tacc, grow, it.abs_m * BM + row, count);
+                } else if (it.type == OP_COND) {
+                    // c = acc + bc stays in registers; s_k = SiLU(c + temb_k) leaves as one bf16 slab per step.
+                    // The warp's shared memory holds six such slabs; a slab is reused three stores later.
+                    if (lane == 0) ptx::bulk_wait_read<0>();
+                    __syncwarp();
+                    int n_st = 0;
+#pragma unroll 1
+                    for (int j = 0; j < io.nch && !fail; ++j) {
+                        float cv[32];
+                        load_acc32(tacc + io.acc0 + 32 * j, cv);
+                        add_bias32(cv, P.bc + io.col0 + 32 * j);
+#pragma unroll 1
+                        for (int k = 0; k < P.K; ++k, ++n_st) {
+                            const uint32_t sl = my_buf + (uint32_t)(n_st % 6) * SLAB_H;
+                            if (n_st >= 6) {
+                                if (lane == 0) ptx::bulk_wait_read<5>();
+                                __syncwarp();
+                            }
+                            float sv[32];
+                            const float* tb = P.temb + (size_t)k * P.W + io.col0 + 32 * j;
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                const float4 t4 = __ldg(reinterpret_cast<const float4*>(tb + i));
+                                sv[i] = silu_f(cv[i] + t4.x); sv[i + 1] = silu_f(cv[i + 1] + t4.y);
+                                sv[i + 2] = silu_f(cv[i + 2] + t4.z); sv[i + 3] = silu_f(cv[i + 3] + t4.w);
+                            }
+                            slabH_write(sl, lane, sv);
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                ptx::tma_store_2d(P.maps + EMAP_S, sl, io.col0 + 32 * j, k * P.R + row0);
+                                ptx::bulk_commit();
+                            }
+                        }
+                    }
                 } else {
                     Stats st;
                     st.init(0.f);
@@ -1009,14 +1054,14 @@ inline float bf16_bits_to_float(uint16_t b) {
 struct ardiff_head {
     ardiff_head_desc d;
     int device, n_sm, grid, coop;
-    int NT, TGu, slots, T_pro, T_step, C_pro, C_step, gcnt[2], n_phases;
+    int NT, TGu, slots, T_pro, T_step, C_pro, C_step, n_phases;
     int64_t max_tiles;
     std::vector<void*> allocs;
     // device
     bf16 *Wcat, *Wc, *Win, *Wt1, *Wt2;
     float *bias_cat, *bc, *bin, *bt1, *bt2, *temb, *temb_hidden;
     bf16 *z, *xb, *s, *u, *a, *g0, *g1;
-    float *x, *c, *h;
+    float *x, *h;
     float2* stats;
     int *counters, *status;  // status[0] = status word, status[1] = abort flag
     long long* trace;        // per-item time stamps (only with ARDIFF_HEAD_PROFILE)
@@ -1104,12 +1149,10 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     const int W = d.W, C = d.C, Dc = d.Dc, L = d.L;
     const int NT = W / BN;
     H->NT = NT;
-    H->T_pro = 1 + NT;
+    H->T_pro = 1 + 2 * NT;     // gather, conditioning items, the gate of step 0 / block 0
     H->T_step = NT * (3 + 5 * L) + 1;
     H->C_pro = 1 + NT;
     H->C_step = NT * (3 + 4 * L) + 1;
-    H->gcnt[0] = NT * ((L + 1) / 2);
-    H->gcnt[1] = NT * (L / 2);
     H->max_tiles = (d.max_tokens + BM - 1) / BM;
     if (H->max_tiles < 1) H->max_tiles = 1;
 
@@ -1214,13 +1257,12 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     // ---- scratch ----
     TRY(dev_alloc(H, &H->z, R * Dc, true));
     TRY(dev_alloc(H, &H->xb, R * XB_COLS, true));  // columns >= C stay zero for ever
-    TRY(dev_alloc(H, &H->s, R * W, true));
+    TRY(dev_alloc(H, &H->s, (size_t)kmax * R * W, true));   // s_k for every step, [k][row][W]
     TRY(dev_alloc(H, &H->u, R * W, true));
     TRY(dev_alloc(H, &H->a, R * W, true));
     TRY(dev_alloc(H, &H->g0, R * W, true));
     TRY(dev_alloc(H, &H->g1, R * W, true));
     TRY(dev_alloc(H, &H->x, R * C, true));
-    TRY(dev_alloc(H, &H->c, R * W, true));
     TRY(dev_alloc(H, &H->h, R * W, true));
     TRY(dev_alloc(H, &H->stats, R * 2 * NT, true));
     TRY(dev_alloc(H, &H->counters, ((size_t)H->max_tiles + 2) * CTRS, true));
@@ -1233,29 +1275,33 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     {
         std::vector<Phase> ph;
         int cum = 0;
-        auto add = [&](int type, int block, int tile0, int ntiles, size_t b_row0, int offA, int gsel, int goff) {
+        auto add = [&](int type, int block, int tile0, int ntiles, size_t b_row0, int offA, int kplus) {
             if (ntiles <= 0) return;
-            ph.push_back(Phase{type, block, tile0, ntiles, cum, (int)b_row0, offA, gsel, goff});
+            ph.push_back(Phase{type, block, tile0, ntiles, cum, (int)b_row0, offA, kplus});
             cum += ntiles;
         };
-        auto gate = [&](int b, int tile0, int ntiles) {
-            // needs s of this step (the in-projection items) and its buffer, last read by block b-2
-            const int offA = NT + (b >= 2 ? 4 * NT * (b - 1) : 0);
-            add(OP_GATE, b, tile0, ntiles, b * blk_rows + 2 * (size_t)W, offA, 1 + (b & 1), 0);
+        // A gate only needs s (known from the start of the call) and its buffer, last read by the block two
+        // gates earlier: chain items of the blocks before `host` must be complete.
+        auto gate = [&](int b, int kplus, int host, int tile0, int ntiles) {
+            add(OP_GATE, b, tile0, ntiles, b * blk_rows + 2 * (size_t)W, NT + 4 * NT * host, kplus);
         };
-        const int na = NT / 2;   // gate tiles of the next block placed between G1 and G2; the rest follow G2
-        add(OP_IN, -1, 0, NT, 0, 0, 0, 0);
-        gate(0, 0, NT);
+        const int na = NT / 2;
+        add(OP_IN, -1, 0, NT, 0, 0, 0);
         for (int b = 0; b < L; ++b) {
             const int base = NT + 4 * NT * b;
-            add(OP_SS, b, 0, 2 * NT, b * blk_rows, base, 0, 0);
-            add(OP_G1, b, 0, NT, b * blk_rows + 3 * (size_t)W, base + 2 * NT, 0, 0);
-            if (b + 1 < L) gate(b + 1, 0, na);
-            add(OP_G2, b, 0, NT, b * blk_rows + 4 * (size_t)W, base + 3 * NT, 1 + (b & 1), NT * ((b >> 1) + 1));
-            if (b + 1 < L) gate(b + 1, na, NT - na);
+            add(OP_SS, b, 0, 2 * NT, b * blk_rows, base, 0);
+            add(OP_G1, b, 0, NT, b * blk_rows + 3 * (size_t)W, base + 2 * NT, 0);
+            // block b hosts the gate of the next block: half between its two dependent GEMMs, half after
+            if (b + 1 < L) gate(b + 1, 0, b, 0, na);
+            add(OP_G2, b, 0, NT, b * blk_rows + 4 * (size_t)W, base + 3 * NT, 0);
+            if (b + 1 < L) gate(b + 1, 0, b, na, NT - na);
         }
-        add(OP_FSS, -1, 0, 2 * NT, fm_row0, NT + 4 * NT * L, 0, 0);
-        add(OP_OUT, -1, 0, 1, out_row0, NT + 4 * NT * L + 2 * NT, 0, 0);
+        // the last block hosts the first gate of the NEXT step, spread over the step boundary where the chain
+        // (final modulation -> out-projection -> in-projection) has little else to overlap with
+        add(OP_FSS, -1, 0, 2 * NT, fm_row0, NT + 4 * NT * L, 0);
+        gate(0, 1, L - 1, 0, na);
+        add(OP_OUT, -1, 0, 1, out_row0, NT + 4 * NT * L + 2 * NT, 0);
+        gate(0, 1, L - 1, na, NT - na);
         if (cum != H->T_step) {
             free_all(H);
             delete H;
@@ -1277,7 +1323,7 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         bool ok = true;
         ok &= make_map(&maps[MAP_Z], H->z, R, Dc, BM);
         ok &= make_map(&maps[MAP_XB], H->xb, R, XB_COLS, BM);
-        ok &= make_map(&maps[MAP_S], H->s, R, W, BM);
+        ok &= make_map(&maps[MAP_S], H->s, (uint64_t)kmax * R, W, BM);
         ok &= make_map(&maps[MAP_U], H->u, R, W, BM);
         ok &= make_map(&maps[MAP_A], H->a, R, W, BM);
         // a CTA of a pair stages half of the weight tile's rows
@@ -1286,8 +1332,7 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, B_ROWS);
         ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C / 2);
         ok &= make_slab_map(&maps[EMAP_H], H->h, R, W, true);
-        ok &= make_slab_map(&maps[EMAP_C], H->c, R, W, true);
-        ok &= make_slab_map(&maps[EMAP_S], H->s, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_S], H->s, (uint64_t)kmax * R, W, false);
         ok &= make_slab_map(&maps[EMAP_U], H->u, R, W, false);
         ok &= make_slab_map(&maps[EMAP_A], H->a, R, W, false);
         ok &= make_slab_map(&maps[EMAP_G0], H->g0, R, W, false);
@@ -1359,12 +1404,12 @@ int head_sample_impl(const ardiff_head* H, const void* cond, const float* noise,
     P.C = C; P.Dc = H->d.Dc; P.W = W; P.L = H->d.L; P.K = K; P.NT = H->NT; P.TGu = H->TGu; P.slots = H->slots;
     P.T_pro = H->T_pro; P.T_step = H->T_step; P.T_chain = H->T_pro + K * H->T_step;
     P.C_pro = H->C_pro; P.C_step = H->C_step; P.C_total = H->C_pro + K * H->C_step;
-    P.gcnt[0] = H->gcnt[0]; P.gcnt[1] = H->gcnt[1];
+    P.R = H->slots * BM;
     P.max_tokens = (int)H->d.max_tokens;
     P.phases = H->phases; P.cum2phase = H->cum2phase; P.maps = H->maps;
     P.cond = reinterpret_cast<const bf16*>(cond); P.noise = noise; P.idx = idx; P.count = count; P.out = out;
     P.z = H->z; P.xb = H->xb; P.s = H->s; P.u = H->u; P.a = H->a; P.g0 = H->g0; P.g1 = H->g1;
-    P.x = H->x; P.c = H->c; P.h = H->h; P.stats = H->stats;
+    P.x = H->x; P.h = H->h; P.stats = H->stats;
     P.bias_cat = H->bias_cat; P.bc = H->bc; P.bin = H->bin; P.temb = H->temb;
     P.counters = H->counters; P.status = H->status; P.abort_flag = H->status + 1;
     P.trace = H->trace;
@@ -1467,7 +1512,6 @@ extern "C" void* ardiff_head_debug_ptr(ardiff_head* H, const char* name) {
     if (!strcmp(name, "g0")) return H->g0;
     if (!strcmp(name, "g1")) return H->g1;
     if (!strcmp(name, "x")) return H->x;
-    if (!strcmp(name, "c")) return H->c;
     if (!strcmp(name, "h")) return H->h;
     if (!strcmp(name, "temb")) return H->temb;
     if (!strcmp(name, "counters")) return H->counters;
