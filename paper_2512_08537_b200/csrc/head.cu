@@ -536,26 +536,39 @@ __device__ __forceinline__ void epi_out(const HeadParams& P, const Item& it, uin
 }
 
 // 16 rows of this token tile per epilogue warp: z = cond[idx[j]], x = noise[idx[j]], xb = bf16(x);
-// rows past count: 0
+// rows past count: 0. The 16 token ids are fetched with one load and the rows are copied four at a
+// time, so that many independent loads are in flight (the rows sit in HBM).
 __device__ __forceinline__ void gather_rows(const HeadParams& P, const Item& it, int ew, int lane, int count) {
     const int chunks = P.Dc / 8;  // 16-byte chunks per cond row
     constexpr int RPW = BM / EPI_WARPS;
-    for (int r = ew * RPW; r < ew * RPW + RPW; ++r) {
-        const int j = it.abs_m * BM + r;
-        const int grow = it.slot_row0 + r;
-        const bool valid = j < count;
-        const size_t tok = valid ? (size_t)__ldg(P.idx + j) : 0;
-        const uint4* src = reinterpret_cast<const uint4*>(P.cond + tok * P.Dc);
-        uint4* dst = reinterpret_cast<uint4*>(P.z + (size_t)grow * P.Dc);
+    const int r0 = ew * RPW;
+    const int j0 = it.abs_m * BM + r0;
+    int my_tok = -1;
+    if (lane < RPW && j0 + lane < count) my_tok = __ldg(P.idx + j0 + lane);
+#pragma unroll 1
+    for (int rr = 0; rr < RPW; rr += 4) {
+        int tok[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tok[q] = __shfl_sync(0xffffffffu, my_tok, rr + q);
         for (int c = lane; c < chunks; c += 32) {
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (valid) v = __ldg(src + c);
-            dst[c] = v;
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                v[q] = make_uint4(0, 0, 0, 0);
+                if (tok[q] >= 0) v[q] = __ldg(reinterpret_cast<const uint4*>(P.cond + (size_t)tok[q] * P.Dc) + c);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                reinterpret_cast<uint4*>(P.z + (size_t)(it.slot_row0 + r0 + rr + q) * P.Dc)[c] = v[q];
         }
         for (int c = lane; c < P.C; c += 32) {
-            const float xv = valid ? __ldg(P.noise + tok * P.C + c) : 0.f;
-            P.x[(size_t)grow * P.C + c] = xv;
-            P.xb[(size_t)grow * XB_COLS + c] = __float2bfloat16_rn(xv);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int grow = it.slot_row0 + r0 + rr + q;
+                const float xv = tok[q] >= 0 ? __ldg(P.noise + (size_t)tok[q] * P.C + c) : 0.f;
+                P.x[(size_t)grow * P.C + c] = xv;
+                P.xb[(size_t)grow * XB_COLS + c] = __float2bfloat16_rn(xv);
+            }
         }
     }
 }
