@@ -249,6 +249,7 @@ int ardiff_head_last_kernel_ms(ardiff_head* head, float* ms);
  *   feat   host bf16 [n][d],  cond host bf16 [n][Dc],  noise host float [n][C]
  *   out    host float [n][C]: rows of kept tokens hold the sample, dropped rows are 0
  *   mask   host uint8 [n],    count host int32 [1]
+ * With n == 0 the five batch pointers may be NULL (count is still written).
  * The call waits for `stream` before it returns, so the host outputs are valid on return.
  * ------------------------------------------------------------------------------------- */
 typedef struct ardiff_pipeline ardiff_pipeline;
@@ -258,6 +259,45 @@ int ardiff_pipeline_destroy(ardiff_pipeline* pipeline);
 int ardiff_pipeline_run_host(ardiff_pipeline* pipeline, const void* feat, const void* cond,
                              const float* noise, int64_t n, float tau, const float* t_sched, int32_t K,
                              float* out, uint8_t* mask, int32_t* count, void* stream);
+
+/* Overlapped form of the same path, for a stream of batches. A pipeline created with
+ * ardiff_pipeline_create_slots(..., n_slots >= 2, ...) owns n_slots sets of device staging
+ * buffers and three streams (copy-in, compute, copy-out), so the host->device copy of one batch
+ * and the device->host copy of another run under the kernels of a third. (The paper describes
+ * no host interface; this is packaging around the path of Sec. 3.2-3.3.)
+ *
+ *   ardiff_pipeline_submit  enqueues copy-in, gate, head and copy-out of one batch on `slot`
+ *                           (0 <= slot < n_slots) and returns without waiting. Arguments as for
+ *                           ardiff_pipeline_run_host; t_sched is read before the call returns,
+ *                           every other host buffer must stay valid (and, for the copies to be
+ *                           asynchronous, pinned) until ardiff_pipeline_wait(slot) has returned.
+ *                           The batch starts after the work `stream` holds at the time of the
+ *                           call; nothing else is enqueued on `stream`. Re-using a slot is ordered
+ *                           on the device after the slot's previous batch; the HOST buffers of that
+ *                           previous batch are the caller's to keep apart (wait first, or use others).
+ *   ardiff_pipeline_wait    blocks the host until the batch last submitted on `slot` has been
+ *                           copied out, stores its number of kept tokens in that submission's
+ *                           `count` (only this call writes it: the pipeline stages the value in
+ *                           pinned memory of its own so that a pageable `count` cannot stall the
+ *                           submitting thread) and returns what that submission returned. A slot never
+ *                           submitted to returns ARDIFF_OK at once.
+ *   ardiff_pipeline_join    makes `stream` wait (on the device) for every batch submitted so far;
+ *                           the host does not block.
+ *
+ * Batches run through the head in submission order. Calls on one pipeline must come from one
+ * host thread at a time. ardiff_pipeline_create gives a one-slot pipeline, on which these three
+ * calls return ARDIFF_ERR_UNSUPPORTED; ardiff_pipeline_run_host works on any pipeline and uses
+ * slot 0 (it first waits for a batch still in flight there). Errors: ARDIFF_ERR_NULL,
+ * ARDIFF_ERR_SHAPE (slot or n out of range), ARDIFF_ERR_CUDA, and whatever the gate or the head
+ * return; after a failed submit the slot's events are still recorded, so wait never hangs. */
+#define ARDIFF_PIPELINE_MAX_SLOTS 4
+int ardiff_pipeline_create_slots(ardiff_head* head, int64_t max_n, int32_t d, int32_t Dc, int32_t C,
+                                 int32_t n_slots, ardiff_pipeline** pipeline_out);
+int ardiff_pipeline_submit(ardiff_pipeline* pipeline, int32_t slot, const void* feat, const void* cond,
+                           const float* noise, int64_t n, float tau, const float* t_sched, int32_t K,
+                           float* out, uint8_t* mask, int32_t* count, void* stream);
+int ardiff_pipeline_wait(ardiff_pipeline* pipeline, int32_t slot);
+int ardiff_pipeline_join(ardiff_pipeline* pipeline, void* stream);
 
 /* Number of kernel launches the last ardiff_head_sample / ardiff_entropy_gate call on this
  * thread enqueued (for launch accounting by benchmarks). */

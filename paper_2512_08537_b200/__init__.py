@@ -305,14 +305,19 @@ class Head:
 
 
 class Pipeline:
-    """Host-buffer front end (ardiff_pipeline_*): device staging for up to max_n tokens."""
+    """Host-buffer front end (ardiff_pipeline_*): device staging for up to max_n tokens.
 
-    def __init__(self, head: Head, max_n: int, d: int):
+    With slots >= 2 the overlapped calls (ardiff_pipeline_submit / _wait / _join) are available."""
+
+    def __init__(self, head: Head, max_n: int, d: int, slots: int = 1):
         self.head = head
         self.d, self.Dc, self.C = d, head.desc.Dc, head.desc.C
+        self.slots = slots
+        self._counts = [ctypes.c_int32(0) for _ in range(slots)]
         p = ctypes.c_void_p()
-        _check(lib().ardiff_pipeline_create(head._h, max_n, d, self.Dc, self.C, ctypes.byref(p)),
-               "ardiff_pipeline_create")
+        vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+        fn = _fn("ardiff_pipeline_create_slots", [vp, i64, i32, i32, i32, i32, ctypes.POINTER(vp)])
+        _check(fn(head._h, max_n, d, self.Dc, self.C, slots, ctypes.byref(p)), "ardiff_pipeline_create_slots")
         self._p = p
 
     def ardiff_pipeline_run_host(self, feat, cond, noise, tau, t_sched, out, mask, stream=None) -> int:
@@ -327,6 +332,31 @@ class Pipeline:
                                             mask.data_ptr(), ctypes.addressof(count), _stream_ptr(stream))
         _check(rc, "ardiff_pipeline_run_host")
         return int(count.value)
+
+    def ardiff_pipeline_submit(self, slot: int, feat, cond, noise, tau, t_sched, out, mask, stream=None) -> None:
+        """Enqueue one batch on `slot` without waiting; the host tensors must stay alive (and should
+        be pinned) until ardiff_pipeline_wait(slot)."""
+        import numpy as np
+        ts = np.ascontiguousarray(t_sched, dtype=np.float32)
+        vp, i64, i32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float
+        fn = _fn("ardiff_pipeline_submit", [vp, i32, vp, vp, vp, i64, f32, vp, i32, vp, vp, vp, vp])
+        if not 0 <= slot < self.slots:
+            raise ValueError("slot out of range")
+        rc = fn(self._p, slot, feat.data_ptr(), cond.data_ptr(), noise.data_ptr(), feat.shape[0], float(tau),
+                ts.ctypes.data, ts.shape[0] - 1, out.data_ptr(), mask.data_ptr(),
+                ctypes.addressof(self._counts[slot]), _stream_ptr(stream))
+        _check(rc, "ardiff_pipeline_submit")
+
+    def ardiff_pipeline_wait(self, slot: int) -> int:
+        """Block until the batch on `slot` has been copied out; returns its number of kept tokens."""
+        fn = _fn("ardiff_pipeline_wait", [ctypes.c_void_p, ctypes.c_int32])
+        _check(fn(self._p, slot), "ardiff_pipeline_wait")
+        return int(self._counts[slot].value)
+
+    def ardiff_pipeline_join(self, stream=None) -> None:
+        """Make `stream` wait on the device for every batch submitted so far."""
+        fn = _fn("ardiff_pipeline_join", [ctypes.c_void_p, ctypes.c_void_p])
+        _check(fn(self._p, _stream_ptr(stream)), "ardiff_pipeline_join")
 
     def close(self):
         if getattr(self, "_p", None) is not None and self._p:
