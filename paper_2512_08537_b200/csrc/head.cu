@@ -359,12 +359,11 @@ __device__ __forceinline__ void load_acc32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ void add_bias32(float (&v)[32], const float* __restrict__ bias) {
+// The chunk's 32 bias values sit one per lane (fetched at the start of the item, while the accumulator is still
+// being produced) and are handed round by shuffle: no global load on the chunk's critical path.
+__device__ __forceinline__ void add_bias32(float (&v)[32], float b_lane) {
 #pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        const float4 b = __ldg(reinterpret_cast<const float4*>(bias + i));
-        v[i] += b.x; v[i + 1] += b.y; v[i + 2] += b.z; v[i + 3] += b.w;
-    }
+    for (int i = 0; i < 32; ++i) v[i] += __shfl_sync(0xffffffffu, b_lane, i);
 }
 
 __device__ __forceinline__ void slabF_read(uint32_t base, int r, float (&v)[32]) {
@@ -425,12 +424,12 @@ __device__ __forceinline__ void row_mean_rstd(const HeadParams& P, int grow, flo
 // for the 256-column ops), bufF / bufH: this warp's slabs for the chunk; r: lane.
 __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, uint32_t acc, int acc_col, int col,
                                           bool first, uint32_t bufF, uint32_t bufH, int r, Stats& st, float mean,
-                                          float rstd) {
+                                          float rstd, float b0, float b1) {
     float v[32];
     switch (it.type) {
         case OP_IN: {                         // h = acc + bin
             load_acc32(acc, v);
-            add_bias32(v, P.bin + col);
+            add_bias32(v, b0);
             if (first) st.init(v[0]);
 #pragma unroll
             for (int i = 0; i < 32; ++i) st.add(v[i]);
@@ -439,12 +438,11 @@ __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, u
         }
         case OP_SS:
         case OP_FSS: {                        // u = LN(h) * (1 + scale) + shift
-            const float* bias = P.bias_cat + it.b_row + acc_col;
             float sc[32], hv[32];
             load_acc32(acc, v);
             load_acc32(acc + 128, sc);
-            add_bias32(v, bias);
-            add_bias32(sc, bias + 128);
+            add_bias32(v, b0);
+            add_bias32(sc, b1);
             slabF_read(bufF, r, hv);
 #pragma unroll
             for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], v[i]);
@@ -453,13 +451,13 @@ __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, u
         }
         case OP_GATE: {                       // g = acc + bias
             load_acc32(acc, v);
-            add_bias32(v, P.bias_cat + it.b_row + acc_col);
+            add_bias32(v, b0);
             slabH_write(bufH, r, v);
             break;
         }
         case OP_G1: {                         // a = SiLU(acc + b1)
             load_acc32(acc, v);
-            add_bias32(v, P.bias_cat + it.b_row + acc_col);
+            add_bias32(v, b0);
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = silu_f(v[i]);
             slabH_write(bufH, r, v);
@@ -468,7 +466,7 @@ __device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, u
         default: {                            // OP_G2: h += g * (acc + b2)
             float gv[32], hv[32];
             load_acc32(acc, v);
-            add_bias32(v, P.bias_cat + it.b_row + acc_col);
+            add_bias32(v, b0);
             slabH_read(bufH, r, gv);
             slabF_read(bufF, r, hv);
 #pragma unroll
@@ -812,6 +810,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                     ld_pending |= 1u << b;
                 };
                 if (has_loads && io.nch > 0) issue_load(0);
+                // bias values of the warp's chunks, one column per lane (modulation items: shift in bq[0..1], scale in bq[2..3])
+                float bq[4] = {0.f, 0.f, 0.f, 0.f};
+                {
+                    const bool mod = (it.type == OP_SS || it.type == OP_FSS);
+                    const float* bb = it.type == OP_IN     ? P.bin + io.col0
+                                      : it.type == OP_COND ? P.bc + io.col0
+                                                           : P.bias_cat + it.b_row + io.acc0;
+                    if (it.type != OP_OUT) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            bq[q] = __ldg(bb + (mod ? (q & 1) * 32 + (q >> 1) * 128 : q * 32) + lane);
+                    }
+                }
                 const int grow = it.slot_row0 + row;
                 float mean = 0.f, rstd = 0.f;
                 if (it.type == OP_SS || it.type == OP_FSS) row_mean_rstd(P, grow, mean, rstd);
@@ -835,22 +846,20 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                     for (int j = 0; j < io.nch && !fail; ++j) {
                         float cv[32];
                         load_acc32(tacc + io.acc0 + 32 * j, cv);
-                        add_bias32(cv, P.bc + io.col0 + 32 * j);
+                        add_bias32(cv, j == 0 ? bq[0] : j == 1 ? bq[1] : j == 2 ? bq[2] : bq[3]);
+                        float tk = __ldg(P.temb + io.col0 + 32 * j + lane);          // temb_k of this lane's column
 #pragma unroll 1
                         for (int k = 0; k < P.K; ++k, ++n_st) {
+                            const float tcur = tk;
+                            if (k + 1 < P.K) tk = __ldg(P.temb + (size_t)(k + 1) * P.W + io.col0 + 32 * j + lane);
                             const uint32_t sl = my_buf + (uint32_t)(n_st % 6) * SLAB_H;
                             if (n_st >= 6) {
                                 if (lane == 0) ptx::bulk_wait_read<5>();
                                 __syncwarp();
                             }
                             float sv[32];
-                            const float* tb = P.temb + (size_t)k * P.W + io.col0 + 32 * j;
 #pragma unroll
-                            for (int i = 0; i < 32; i += 4) {
-                                const float4 t4 = __ldg(reinterpret_cast<const float4*>(tb + i));
-                                sv[i] = silu_f(cv[i] + t4.x); sv[i + 1] = silu_f(cv[i + 1] + t4.y);
-                                sv[i + 2] = silu_f(cv[i + 2] + t4.z); sv[i + 3] = silu_f(cv[i + 3] + t4.w);
-                            }
+                            for (int i = 0; i < 32; ++i) sv[i] = silu_f(cv[i] + __shfl_sync(0xffffffffu, tcur, i));
                             slabH_write(sl, lane, sv);
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
@@ -884,8 +893,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                             if (lane == 0) ptx::bulk_wait_read<EPI_NB - 1>();
                             __syncwarp();
                         }
+                        const float b0 = j == 0 ? bq[0] : j == 1 ? bq[1] : j == 2 ? bq[2] : bq[3];
+                        const float b1 = j == 0 ? bq[2] : bq[3];        // modulation items: the scale's bias
                         epi_chunk(P, it, tacc + io.acc0 + 32 * j, io.acc0 + 32 * j, io.col0 + 32 * j, j == 0, bufF, bufH,
-                                  lane, st, mean, rstd);
+                                  lane, st, mean, rstd, b0, b1);
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
