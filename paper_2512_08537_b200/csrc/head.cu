@@ -664,7 +664,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             TRACE(0, 0);
             if (lane == 0) ptx::mbar_arrive(dep_bar(seq));      // the epilogue may now load this item's slabs
             ++seq;
-            ptx::fence_proxy_async();
+            // operands that other CTAs wrote with plain stores (z, xb) cross from the generic to the async proxy;
+            // everything else was written by TMA stores and is read by TMA loads
+            if (it.type == OP_COND || it.type == OP_IN) ptx::fence_proxy_async();
             const void* map_a = P.maps + it.map_a;
             const void* map_b = P.maps + it.map_b;
             const int b_rows = it.umma_n / 2;                         // rows of B this CTA stages
@@ -796,7 +798,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 if (ew == 0) TRACE(2, 0);
                 const EpiIO io = epi_io(it, half);
                 const bool has_loads = (io.ldF >= 0) || (io.ldH >= 0);
-                if (has_loads) ptx::fence_proxy_async();   // other CTAs' writes -> this warp's TMA reads
+                // h and the gate values were written by TMA stores and are read by TMA loads: no proxy is crossed
                 const int row0 = it.slot_row0 + quarter * 32;
                 auto issue_load = [&](int j) {
                     const int b = j & 1;
