@@ -30,7 +30,7 @@ METRIC = "gated draft tokens/sec through K-step head"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 512 << 20
 # dram bytes per launch of the head kernel from the ncu capture summarised under profiles/
-TRAFFIC_BYTES = {"cfg2": 4.137e9}
+TRAFFIC_BYTES = {"cfg2": 4.125e9}
 
 
 def peaks():
