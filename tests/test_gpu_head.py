@@ -147,6 +147,40 @@ def test_two_calls_on_one_head_give_identical_results():
     head.close()
 
 
+@pytest.mark.parametrize("name,runs,K", [("cfg2", 12, 4), ("cfg3", 4, 2)])
+def test_full_size_runs_are_bit_identical(name, runs, K):
+    """The kernel's arithmetic has a fixed order, so equal inputs must give equal bits however the
+    items of the many CTAs interleave. A tile read before its producer's writes were visible (an
+    ordering bug between CTAs) shows up here as a run that differs; the cache flush and the
+    varying survivor counts in between change the timing from run to run."""
+    dev = require_cuda()
+    wl = synth.workload(name, K=K)
+    w, t = synth.head_weights(wl), synth.t_sched(wl.K)
+    cond, noise = dev_bf16(synth.cond(wl)), dev_f32(synth.noise(wl))
+    head = make_head(wl, w)
+    S = int(round(wl.n * (1 - wl.filter_q)))
+    idx = torch.randperm(wl.n, device=dev, generator=torch.Generator(device=dev).manual_seed(3))[:S]
+    idx = idx.sort().values.to(torch.int32).contiguous()
+    count = torch.tensor([S], dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    ref = None
+    for r in range(runs):
+        if r % 3 == 1:                                  # a different, smaller run in between
+            c2 = torch.tensor([S // 2 + 7 * r], dtype=torch.int32, device=dev)
+            scratch = torch.empty((wl.n, wl.C), dtype=torch.float32, device=dev)
+            head.ardiff_head_sample(cond, noise, t, idx, c2, scratch)
+        flush.fill_(r)
+        out = torch.full((wl.n, wl.C), SENTINEL, dtype=torch.float32, device=dev)
+        head.ardiff_head_sample(cond, noise, t, idx, count, out)
+        assert head.status() == 0
+        if ref is None:
+            ref = out
+        else:
+            assert torch.equal(out, ref), f"run {r} differs from run 0"
+    assert bool(torch.isfinite(ref[idx.long()]).all())
+    head.close()
+
+
 @pytest.mark.parametrize("name,extra", [("cfg2", 160), ("cfg3", 48), ("cfg4", 32)])
 def test_workload_configs_sampled_tokens(name, extra):
     """Full-size gate -> head run; the oracle checks the first, a middle and the last (ragged)
