@@ -181,12 +181,14 @@ def test_full_size_runs_are_bit_identical(name, runs, K):
     head.close()
 
 
-@pytest.mark.parametrize("name,extra", [("cfg2", 160), ("cfg3", 48), ("cfg4", 32)])
-def test_workload_configs_sampled_tokens(name, extra):
+@pytest.mark.parametrize("name,extra,K", [("cfg2", 160, None), ("cfg3", 48, None), ("cfg4", 32, None),
+                                          ("cfg3", 24, 1), ("cfg3", 12, 8)])
+def test_workload_configs_sampled_tokens(name, extra, K):
     """Full-size gate -> head run; the oracle checks the first, a middle and the last (ragged)
-    token tile plus random survivors one by one (tokens are independent)."""
+    token tile plus random survivors one by one (tokens are independent). cfg 3 also runs at the
+    other step counts its workload names (K = 1 and 8)."""
     dev = require_cuda()
-    wl = synth.workload(name)
+    wl = synth.workload(name) if K is None else synth.workload(name, K=K)
     feat_bits = synth.features(wl)
     H = oracle.entropy(feat_bits)
     Hs = np.sort(H)
@@ -203,7 +205,8 @@ def test_workload_configs_sampled_tokens(name, extra):
     got = out.cpu().numpy()
     if name != "cfg2":                      # keep the oracle's share of the run to seconds
         pos = sample_tokens(idx_h, extra=extra)
-        pos = np.concatenate([pos[:16], pos[len(pos) // 2: len(pos) // 2 + 8], pos[-16:],
+        edge = 16 if K is None else 6
+        pos = np.concatenate([pos[:edge], pos[len(pos) // 2: len(pos) // 2 + edge // 2], pos[-edge:],
                               np.random.default_rng(1).choice(pos, size=extra, replace=False)])
         pos = np.unique(pos)
     else:
