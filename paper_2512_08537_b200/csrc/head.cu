@@ -18,6 +18,11 @@
 // are placed between the dependent phases of block b, where they cover the latency of the chain.
 // Dependencies between items are tracked per token tile by three counters (chain, gates of even
 // blocks, gates of odd blocks) with release/acquire at gpu scope; every wait is bounded.
+// The binding resource is the SM's shared-memory bandwidth (about 128 B/clk): at tensor peak the operand
+// ring alone takes all of it (32 KB written by TMA and 32 KB read by the MMA per 512-cycle stage), and every
+// byte an epilogue stages in a slab is paid twice. Hence biases travel in registers (one column per lane,
+// handed round by shuffle), c never leaves the accumulator, and proxy fences sit only where a proxy is
+// really crossed: a fence in the producer's path stalls the whole ring.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
