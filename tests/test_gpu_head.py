@@ -222,6 +222,39 @@ def test_workload_configs_sampled_tokens(name, extra, K):
     head.close()
 
 
+def test_two_heads_on_two_streams():
+    """Two heads of different shapes, driven from two streams without any ordering between them: every
+    launch needs the whole GPU (cooperative launch), so the launches take turns; both results must
+    match what each head gives alone."""
+    dev = require_cuda()
+    wa, wb = synth.workload("cfg1", n=700), synth.workload("cfg1", n=900, W=512, L=3, seed=77)
+    outs = {}
+    heads = {}
+    for key, wl in (("a", wa), ("b", wb)):
+        w, t = synth.head_weights(wl), synth.t_sched(wl.K)
+        head = make_head(wl, w)
+        cond, noise = dev_bf16(synth.cond(wl)), dev_f32(synth.noise(wl))
+        idx = torch.arange(wl.n, dtype=torch.int32, device=dev)
+        count = torch.tensor([wl.n], dtype=torch.int32, device=dev)
+        alone = torch.empty((wl.n, wl.C), dtype=torch.float32, device=dev)
+        head.ardiff_head_sample(cond, noise, t, idx, count, alone)
+        heads[key] = (head, cond, noise, t, idx, count, alone, wl)
+    torch.cuda.synchronize()
+    streams = {k: torch.cuda.Stream(device=dev) for k in heads}
+    for rep in range(4):
+        for key, (head, cond, noise, t, idx, count, alone, wl) in heads.items():
+            out = torch.full((wl.n, wl.C), SENTINEL, dtype=torch.float32, device=dev)
+            head.ardiff_head_sample(cond, noise, t, idx, count, out, stream=streams[key])
+            outs[(key, rep)] = out
+    torch.cuda.synchronize()
+    for (key, rep), out in outs.items():
+        head, *_, alone, wl = heads[key]
+        assert head.status() == 0
+        assert torch.equal(out, alone), (key, rep)
+    for head, *_ in heads.values():
+        head.close()
+
+
 def test_bad_arguments_are_rejected():
     require_cuda()
     wl = synth.workload("cfg1")
