@@ -54,7 +54,7 @@ def _load():
         lib.oracle_head_sample_coef.argtypes = [ctypes.POINTER(_HeadParams), vp, vp, vp, i32, vp, vp, i64, vp, i32, vp]
         lib.oracle_gate_blocks.argtypes = [vp, i64, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp]
         lib.oracle_tau_calibrate.argtypes = [vp, i64, vp, vp, vp]
-        lib.oracle_accept_prefix.argtypes = [vp, vp, i64, i32, vp]
+        lib.oracle_accept_prefix.argtypes = [vp, vp, i64, i32, vp, vp]
         lib.oracle_layer_norm.argtypes = [vp, i32, vp]
         lib.oracle_time_embedding.argtypes = [ctypes.POINTER(_HeadParams), ctypes.c_float, vp]
         for f in (lib.oracle_entropy, lib.oracle_gate, lib.oracle_head_sample, lib.oracle_head_sample_coef,
@@ -193,14 +193,20 @@ def tau_calibrate(H: np.ndarray) -> Tuple[float, float, float]:
     return m.value, s.value, t.value
 
 
-def accept_prefix(r: np.ndarray, ratio: np.ndarray, gamma: int) -> np.ndarray:
-    """Accepted draft length per block of gamma: first position whose r exceeds its ratio, else the block length."""
+def accept_prefix(r: np.ndarray, ratio: np.ndarray, gamma: int, block_len: Optional[np.ndarray] = None) -> np.ndarray:
+    """Accepted draft length per block of gamma: first position whose r exceeds its ratio, else the length of
+    the draft (block_len[b] where the early stop truncated the block, the whole block otherwise)."""
     r = np.ascontiguousarray(r, dtype=np.float32)
     ratio = np.ascontiguousarray(ratio, dtype=np.float32)
     n = r.shape[0]
     nb = (n + gamma - 1) // gamma
     out = np.empty((max(nb, 1),), dtype=np.int32)
-    _load().oracle_accept_prefix(r.ctypes.data, ratio.ctypes.data, n, gamma, out.ctypes.data)
+    bl = None
+    if block_len is not None:
+        bl = np.ascontiguousarray(block_len, dtype=np.int32)
+        assert bl.shape == (nb,)
+    _load().oracle_accept_prefix(r.ctypes.data, ratio.ctypes.data, n, gamma,
+                                 bl.ctypes.data if bl is not None else None, out.ctypes.data)
     return out[:nb].copy()
 
 

@@ -130,10 +130,17 @@ void oracle_tau_calibrate(const double* H, int64_t n, double* mean, double* std,
 }
 
 /* Accepted draft length per block (Algorithm 1, Step 4):
- * n_b = min({i-1 : r_i > ratio_i} U {len_b}), i counted from 1 inside the block. */
-void oracle_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma, int32_t* nacc) {
+ * n_b = min({i-1 : r_i > ratio_i} U {len_b}), i counted from 1 inside the block. len_b is
+ * len(draft_tokens) as Step 1 left it: block_len[b] drafts when the early stop truncated the block
+ * (block_len == NULL: nothing was truncated, the whole block reaches Step 4). */
+void oracle_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma, const int32_t* block_len,
+                          int32_t* nacc) {
     for (int64_t b0 = 0, b = 0; b0 < n; b0 += gamma, ++b) {
-        const int64_t b1 = (b0 + gamma < n) ? b0 + gamma : n;
+        int64_t b1 = (b0 + gamma < n) ? b0 + gamma : n;
+        if (block_len) {
+            const int64_t lb = block_len[b] > 0 ? block_len[b] : 0;
+            if (b0 + lb < b1) b1 = b0 + lb;
+        }
         int32_t acc = (int32_t)(b1 - b0);
         for (int64_t i = b0; i < b1; ++i) {
             if (r[i] > ratio[i]) { acc = (int32_t)(i - b0); break; }
@@ -199,7 +206,6 @@ static void time_embedding(const oracle_head_params* P, double t, double* temb, 
     linear(P->Wt2, P->bt2, P->W, P->W, tmpW, temb);
 }
 
-/* One survivor token: K Euler steps of the velocity head. x [C] in/out. */
 /* One survivor token: K steps of the head, each followed by the sampler update
  *   x <- ax_k x + av_k v + an_k z_k        (coef = {ax_0, av_0, an_0, ax_1, ...}, z_k = step noise or none).
  * The Euler flow update is the case ax = 1, av = t_{k+1} - t_k, an = 0. */

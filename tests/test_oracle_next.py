@@ -100,6 +100,43 @@ def test_accept_prefix_brute_force(gamma):
     assert oracle.accept_prefix(eq, eq, 4).tolist() == [4]
 
 
+@pytest.mark.parametrize("gamma", [1, 5, 8])
+def test_accept_prefix_after_early_stop_brute_force(gamma):
+    """Algorithm 1 runs Step 4 on the draft that Step 1 left: len(draft_tokens) is the truncated length, so a
+    rejection at or beyond it is never seen and the accepted count is capped by it."""
+    rng = np.random.default_rng(100 + gamma)
+    n = 131
+    nb = (n + gamma - 1) // gamma
+    r = rng.uniform(0, 1, n).astype(np.float32)
+    ratio = rng.uniform(0.2, 1.4, n).astype(np.float32)
+    full = np.array([min(gamma, n - b * gamma) for b in range(nb)], np.int32)
+    kept = np.minimum(rng.integers(0, gamma + 1, nb).astype(np.int32), full)
+    got = oracle.accept_prefix(r, ratio, gamma, kept)
+    want = []
+    for b in range(nb):
+        draft = range(b * gamma, b * gamma + int(kept[b]))
+        rej = [i - b * gamma for i in draft if r[i] > ratio[i]]
+        want.append(min(rej + [int(kept[b])]))
+    assert got.tolist() == want
+    assert np.all(got <= kept)
+    # no truncation recorded = the untruncated call; an all-rejecting block of kept length 0 accepts nothing
+    assert oracle.accept_prefix(r, ratio, gamma, full).tolist() == oracle.accept_prefix(r, ratio, gamma).tolist()
+    assert oracle.accept_prefix(np.zeros(8, np.float32), np.ones(8, np.float32), 4, np.array([0, 3])).tolist() == [0, 3]
+
+
+def test_early_stop_then_accept_prefix_compose():
+    """Step 1 -> Step 4 as the algorithm writes them: the kept lengths of the block-prefix gate feed the
+    accepted-prefix count; with ratios that never reject, the accepted length is exactly the kept length."""
+    wl = synth.workload("cfg2", n=96)
+    bits = synth.features(wl)
+    H = oracle.entropy(bits)
+    tau = float(np.quantile(H, 0.25))
+    _, _, _, _, ln = oracle.gate_blocks(bits, 1, 8, tau)
+    r = np.full(96, 0.5, np.float32)
+    assert oracle.accept_prefix(r, np.ones(96, np.float32), 8, ln).tolist() == ln.tolist()
+    assert 0 < ln.sum() < 96
+
+
 def test_linear_sampler_with_euler_coefficients_is_the_euler_sampler():
     wl = synth.workload("cfg1", n=40, K=5)
     w, cond, noise = synth.head_weights(wl, std=None), synth.cond(wl), synth.noise(wl)
