@@ -57,9 +57,16 @@ int ardiff_version(void);
  *   entropy (the _ex form) dev float [n] out, or NULL: H_i as computed
  *
  * Rows are read once from HBM (d <= 8192 and d % 8 == 0: registers hold the row; other d
- * take a slower two-pass kernel). Uses a small per-device scratch (per-block counts) that
- * the library allocates on the first call on each device: make that first call outside
- * any stream capture. n == 0 is valid (writes *count = 0).
+ * take a slower two-pass kernel). n == 0 is valid (writes *count = 0).
+ *
+ * Scratch and concurrency. The two kernels of a call hand per-block counts to each other
+ * through a small per-device scratch (512 KB) that the library allocates on the first call on
+ * each device: make that first call outside any stream capture. Every stream gets a slice of
+ * its own, so calls on different streams may overlap on the GPU and calls on one stream are
+ * ordered anyway. The table holds 31 streams per device; calls on any further stream share one
+ * slice and must not overlap each other on the GPU. A call captured into a graph keeps the slice
+ * of the stream it was captured on, whatever stream the graph is later launched on.
+ * ardiff_entropy_gate_ex and ardiff_entropy_gate_blocks use the same scratch under the same rule.
  * ------------------------------------------------------------------------------------- */
 int ardiff_entropy_gate(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask,
                         int32_t* idx, int32_t* count, void* stream);
@@ -82,7 +89,8 @@ int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, float tau, ui
  *   mask, idx, count   as for ardiff_entropy_gate (idx ascending)
  *   block_len      dev int32 [ceil(n / gamma)]  out, or NULL: tokens kept in each block
  * gamma == 1 and rows_per_token == 1 give exactly ardiff_entropy_gate's results.
- * Allocates the same per-device scratch as ardiff_entropy_gate on first use.
+ * n * rows_per_token < 2^31. Allocates and uses the same per-device, per-stream scratch as
+ * ardiff_entropy_gate.
  * ------------------------------------------------------------------------------------- */
 int ardiff_entropy_gate_blocks(const void* feat, int64_t n, int32_t rows_per_token, int32_t d,
                                int32_t gamma, float tau, float* row_entropy, float* token_entropy,
@@ -96,11 +104,15 @@ int ardiff_entropy_gate_blocks(const void* feat, int64_t n, int32_t rows_per_tok
 int ardiff_tau_calibrate(const float* entropy, int64_t n, double* out3, void* stream);
 
 /* Accepted draft length per block (Algorithm 1, Step 4):
- * accepted[b] = min({ i-1 : r_i > ratio_i } U { len_b }), i counted from 1 inside block b.
- *   r, ratio  dev float [n] (the uniform draws and the density ratios p_i/q_i, both supplied by
- *   the caller);  accepted dev int32 [ceil(n / gamma)]. */
-int ardiff_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma, int32_t* accepted,
-                         void* stream);
+ * accepted[b] = min({ i-1 : r_i > ratio_i } U { len_b }), i counted from 1 inside block b, where len_b
+ * is the length of the draft that reaches Step 4, i.e. what Step 1's early stop left of the block.
+ *   r, ratio   dev float [n] (the uniform draws and the density ratios p_i/q_i, both supplied by
+ *              the caller; positions are those of the untruncated blocks of gamma tokens)
+ *   block_len  dev int32 [ceil(n / gamma)], or NULL: tokens of each block that survived Step 1, as
+ *              ardiff_entropy_gate_blocks writes them (NULL: every block is whole)
+ *   accepted   dev int32 [ceil(n / gamma)] */
+int ardiff_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma,
+                         const int32_t* block_len, int32_t* accepted, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * Entropy gate for callers that cannot allocate device memory. (The paper has no counterpart:
@@ -119,7 +131,9 @@ int ardiff_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t 
  * one more limit: n <= ARDIFF_GATE_NOALLOC_MAX_TOKENS, else ARDIFF_ERR_SHAPE and nothing is
  * launched (the fixed number of blocks would otherwise each walk an ever longer token range).
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress,
- * with that device current); make that first call before any stream capture starts.
+ * with that device current), and the first call for each feature-width class (d / 256 rounded up
+ * to 1, 2, 4, 8, 12, 16, 20, 24, 32, or the generic path) loads that kernel and queries its
+ * occupancy: make those first calls before any stream capture starts.
  * All calls on one device share the one array. Every call overwrites the entries it uses
  * before it reads them, so nothing needs clearing between calls and back-to-back calls on one
  * stream are safe; two calls that can run on the GPU at the same time (different streams
@@ -231,20 +245,41 @@ int ardiff_head_sample_coef(const ardiff_head* head, const void* cond, const flo
 
 /* Waits for `stream`, then returns the head's device status word: ARDIFF_OK, or
  * ARDIFF_ERR_TIMEOUT if any bounded wait of an earlier sample call ran out, or
- * ARDIFF_ERR_SHAPE if *count exceeded max_tokens. Clears it. */
+ * ARDIFF_ERR_SHAPE if *count exceeded max_tokens. Clears it. (The status word belongs to the
+ * head, not to a stream: this is the call that reports what the device saw.) */
 int ardiff_head_status(ardiff_head* head, void* stream);
 
-/* Profiling aid: with on != 0, every later ardiff_head_sample on this head records CUDA events
+/* Profiling aids. With on != 0, every later ardiff_head_sample on this head records CUDA events
  * on its stream directly around the persistent head kernel. ardiff_head_last_kernel_ms waits
- * for that kernel and writes its device time in milliseconds (ERR_SHAPE if nothing was timed). */
+ * for that kernel and writes its device time in milliseconds (ERR_SHAPE if nothing was timed).
+ * ardiff_head_last_kernel_clock waits for `stream` and writes the SM clock the last head kernel
+ * really ran at, in MHz: SM cycles divided by wall time, both stamped by one CTA at the start and
+ * the end of the launch (ERR_SHAPE before the first launch).
+ * ardiff_head_set_cooperative(head, 0) launches the head kernel without the cooperative attribute,
+ * for profilers that cannot replay cooperative launches; the kernel and its grid are unchanged, but
+ * the launch no longer fails when the GPU cannot hold the whole grid at once (then waits run into
+ * their bound and ARDIFF_ERR_TIMEOUT is reported). Default: on. */
 int ardiff_head_set_timing(ardiff_head* head, int on);
 int ardiff_head_last_kernel_ms(ardiff_head* head, float* ms);
+int ardiff_head_last_kernel_clock(ardiff_head* head, void* stream, double* sm_mhz);
+int ardiff_head_set_cooperative(ardiff_head* head, int on);
+
+/* Self-test of the bounded device-side waits. Arms the NEXT ardiff_head_sample call on this head:
+ * its dependency waits give up after wait_limit_us microseconds (100 .. 4 000 000) instead of the
+ * default 4 s, and the conditioning tiles of token tile `token_tile` (survivors 128 token_tile ..)
+ * wait for one predecessor more than exists, so that wait runs out. The kernel then raises its
+ * abort flag, every CTA leaves its loops, waits for its own copies in flight, frees its tensor
+ * memory and returns; ardiff_head_status reports ARDIFF_ERR_TIMEOUT and the call's results are
+ * invalid. Nothing faults or traps, and the call after it runs normally. A token_tile beyond the
+ * tiles of that call has no effect. */
+int ardiff_head_inject_stall(ardiff_head* head, int32_t token_tile, uint32_t wait_limit_us);
 
 /* ---------------------------------------------------------------------------------------
  * Host-buffer front end: one call takes a batch that lives in HOST memory through the whole
  * path (copy in, gate, head, copy out). The pipeline object owns device staging buffers for
- * up to max_n tokens of feature width d, conditioning width Dc and token dim C (which must
- * match the head's). Pinned host buffers make the copies asynchronous; pageable ones work too.
+ * up to max_n tokens of feature width d, conditioning width Dc and token dim C (Dc and C must
+ * equal the head's and max_n may not exceed its max_tokens, else ARDIFF_ERR_SHAPE). Pinned host
+ * buffers make the copies asynchronous; pageable ones work too.
  *
  *   feat   host bf16 [n][d],  cond host bf16 [n][Dc],  noise host float [n][C]
  *   out    host float [n][C]: rows of kept tokens hold the sample, dropped rows are 0
@@ -287,7 +322,9 @@ int ardiff_pipeline_run_host(ardiff_pipeline* pipeline, const void* feat, const 
  * Batches run through the head in submission order. Calls on one pipeline must come from one
  * host thread at a time. ardiff_pipeline_create gives a one-slot pipeline, on which these three
  * calls return ARDIFF_ERR_UNSUPPORTED; ardiff_pipeline_run_host works on any pipeline and uses
- * slot 0 (it first waits for a batch still in flight there). Errors: ARDIFF_ERR_NULL,
+ * slot 0: it first waits for a batch still in flight there (delivering its count as
+ * ardiff_pipeline_wait would) and orders its own work on the device after every batch submitted
+ * on the other slots. Errors: ARDIFF_ERR_NULL,
  * ARDIFF_ERR_SHAPE (slot or n out of range), ARDIFF_ERR_CUDA, and whatever the gate or the head
  * return; after a failed submit the slot's events are still recorded, so wait never hangs. */
 #define ARDIFF_PIPELINE_MAX_SLOTS 4

@@ -55,26 +55,25 @@ def lib() -> ctypes.CDLL:
         L.ardiff_entropy_gate.argtypes = [vp, i64, i32, f32, vp, vp, vp, vp]
         L.ardiff_entropy_gate_ex.restype = ctypes.c_int
         L.ardiff_entropy_gate_ex.argtypes = [vp, i64, i32, f32, vp, vp, vp, vp, vp]
-        if hasattr(L, "ardiff_head_create"):
-            L.ardiff_head_create.restype = ctypes.c_int
-            L.ardiff_head_create.argtypes = [ctypes.POINTER(HeadDesc), ctypes.POINTER(HeadHostWeights),
-                                             ctypes.POINTER(vp)]
-            L.ardiff_head_destroy.restype = ctypes.c_int
-            L.ardiff_head_destroy.argtypes = [vp]
-            L.ardiff_head_sample.restype = ctypes.c_int
-            L.ardiff_head_sample.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
-            L.ardiff_head_status.restype = ctypes.c_int
-            L.ardiff_head_status.argtypes = [vp, vp]
-            L.ardiff_head_set_timing.restype = ctypes.c_int
-            L.ardiff_head_set_timing.argtypes = [vp, ctypes.c_int]
-            L.ardiff_head_last_kernel_ms.restype = ctypes.c_int
-            L.ardiff_head_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
-            L.ardiff_pipeline_create.restype = ctypes.c_int
-            L.ardiff_pipeline_create.argtypes = [vp, i64, i32, i32, i32, ctypes.POINTER(vp)]
-            L.ardiff_pipeline_destroy.restype = ctypes.c_int
-            L.ardiff_pipeline_destroy.argtypes = [vp]
-            L.ardiff_pipeline_run_host.restype = ctypes.c_int
-            L.ardiff_pipeline_run_host.argtypes = [vp, vp, vp, vp, i64, f32, vp, i32, vp, vp, vp, vp]
+        L.ardiff_head_create.restype = ctypes.c_int
+        L.ardiff_head_create.argtypes = [ctypes.POINTER(HeadDesc), ctypes.POINTER(HeadHostWeights),
+                                         ctypes.POINTER(vp)]
+        L.ardiff_head_destroy.restype = ctypes.c_int
+        L.ardiff_head_destroy.argtypes = [vp]
+        L.ardiff_head_sample.restype = ctypes.c_int
+        L.ardiff_head_sample.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        L.ardiff_head_status.restype = ctypes.c_int
+        L.ardiff_head_status.argtypes = [vp, vp]
+        L.ardiff_head_set_timing.restype = ctypes.c_int
+        L.ardiff_head_set_timing.argtypes = [vp, ctypes.c_int]
+        L.ardiff_head_last_kernel_ms.restype = ctypes.c_int
+        L.ardiff_head_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+        L.ardiff_pipeline_create.restype = ctypes.c_int
+        L.ardiff_pipeline_create.argtypes = [vp, i64, i32, i32, i32, ctypes.POINTER(vp)]
+        L.ardiff_pipeline_destroy.restype = ctypes.c_int
+        L.ardiff_pipeline_destroy.argtypes = [vp]
+        L.ardiff_pipeline_run_host.restype = ctypes.c_int
+        L.ardiff_pipeline_run_host.argtypes = [vp, vp, vp, vp, i64, f32, vp, i32, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -180,16 +179,21 @@ def ardiff_tau_calibrate(entropy, stream=None):
     return out
 
 
-def ardiff_accept_prefix(r, ratio, gamma: int, stream=None):
-    """Accepted draft length per block of `gamma`: first position with r > ratio, else the block length."""
+def ardiff_accept_prefix(r, ratio, gamma: int, block_len=None, stream=None):
+    """Accepted draft length per block of `gamma`: first position with r > ratio, else the length of the
+    draft (block_len[b] tokens where the early stop truncated block b; the whole block if block_len is None)."""
     import torch
     assert r.is_cuda and r.dtype == torch.float32 and ratio.dtype == torch.float32 and r.shape == ratio.shape
     n = r.numel()
-    out = torch.empty((max((n + gamma - 1) // gamma, 1),), dtype=torch.int32, device=r.device)
+    nb = (n + gamma - 1) // gamma
+    out = torch.empty((max(nb, 1),), dtype=torch.int32, device=r.device)
+    if block_len is not None:
+        assert block_len.is_cuda and block_len.dtype == torch.int32 and block_len.numel() >= nb
     vp = ctypes.c_void_p
-    fn = _fn("ardiff_accept_prefix", [vp, vp, ctypes.c_int64, ctypes.c_int32, vp, vp])
+    fn = _fn("ardiff_accept_prefix", [vp, vp, ctypes.c_int64, ctypes.c_int32, vp, vp, vp])
     with torch.cuda.device(r.device):
-        rc = fn(r.data_ptr(), ratio.data_ptr(), n, gamma, out.data_ptr(), _stream_ptr(stream))
+        rc = fn(r.data_ptr(), ratio.data_ptr(), n, gamma, block_len.data_ptr() if block_len is not None else None,
+                out.data_ptr(), _stream_ptr(stream))
     _check(rc, "ardiff_accept_prefix")
     return out[:(n + gamma - 1) // gamma]
 
@@ -227,8 +231,6 @@ class Head:
                  weights: Dict[str, "object"]):
         import numpy as np
         L_ = lib()
-        if not hasattr(L_, "ardiff_head_create"):
-            raise RuntimeError("libardiff.so was built without the head")
         self.desc = HeadDesc(C=C, Dc=Dc, W=W, L=L, F=F, K_max=K_max, max_tokens=max_tokens)
         keep = {k: np.ascontiguousarray(weights[k]) for k in _WEIGHT_FIELDS}
         for k, a in keep.items():
@@ -291,6 +293,22 @@ class Head:
         ms = ctypes.c_float(0.0)
         _check(lib().ardiff_head_last_kernel_ms(self._h, ctypes.byref(ms)), "ardiff_head_last_kernel_ms")
         return float(ms.value)
+
+    def last_kernel_clock_mhz(self, stream=None) -> float:
+        """SM clock the last head kernel ran at (cycles / wall time, stamped on the device)."""
+        mhz = ctypes.c_double(0.0)
+        fn = _fn("ardiff_head_last_kernel_clock", [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_double)])
+        _check(fn(self._h, _stream_ptr(stream), ctypes.byref(mhz)), "ardiff_head_last_kernel_clock")
+        return float(mhz.value)
+
+    def set_cooperative(self, on: bool):
+        fn = _fn("ardiff_head_set_cooperative", [ctypes.c_void_p, ctypes.c_int])
+        _check(fn(self._h, 1 if on else 0), "ardiff_head_set_cooperative")
+
+    def inject_stall(self, token_tile: int, wait_limit_us: int):
+        """Arms the bounded-wait self-test for the next sample call (see ardiff_head_inject_stall)."""
+        fn = _fn("ardiff_head_inject_stall", [ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32])
+        _check(fn(self._h, token_tile, wait_limit_us), "ardiff_head_inject_stall")
 
     def close(self):
         if getattr(self, "_h", None) is not None and self._h:

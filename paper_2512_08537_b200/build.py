@@ -11,7 +11,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libardiff.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC"]
 
 
 def _nvcc() -> str:
@@ -41,7 +41,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile when the library is missing or older than a source. Returns the library path."""
     if not force and not is_stale():
         return LIB
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = list(NVCC_FLAGS)
     objs = []
     bdir = os.path.join(_HERE, "_build")
     os.makedirs(bdir, exist_ok=True)

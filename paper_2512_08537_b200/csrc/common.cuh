@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "../../include/ardiff.h"
+
 namespace ardiff {
 
 // launches enqueued by the last gate / head call on this host thread
@@ -16,7 +18,11 @@ int gate_launch(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask
 int entropy_rows_launch(const void* feat, int64_t rows, int32_t d, float* entropy, int n_sm, cudaStream_t st);
 int compact_launch(const uint8_t* mask, int64_t n, const int32_t* block_counts, int64_t tokens_per_block, int grid,
                    int32_t* idx, int32_t* count, cudaStream_t st);
-int gate_scratch_get(int32_t** counts, int* max_blocks, int* sms);
+// per-block count scratch of the allocating gate calls: a slice private to `st` on the current device
+int gate_scratch_get(cudaStream_t st, int32_t** counts, int* max_blocks, int* sms);
 int write_zero_count(int32_t* count, cudaStream_t st);
+
+// shape of a head (for callers that must match their buffers to it)
+const ardiff_head_desc* head_desc(const ardiff_head* head);
 
 }  // namespace ardiff

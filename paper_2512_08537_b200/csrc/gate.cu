@@ -18,6 +18,8 @@
 #include <math_constants.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/ardiff.h"
 #include "common.cuh"
 
@@ -275,29 +277,52 @@ compact_kernel(const uint8_t* __restrict__ mask, int64_t n, const int32_t* __res
 
 __global__ void write_zero_count_kernel(int32_t* count) { *count = 0; }
 
-// ---- per-device scratch for the block counts -------------------------------------------------
+// ---- per-device scratch for the block counts: one slice per stream -----------------------------
+// Two gate calls may run on the GPU at the same time only when they were enqueued on different streams,
+// so every stream gets a slice of its own (calls on one stream are ordered and share theirs). The table
+// holds kGateSlices - 1 streams per device; any further stream shares the last slice.
 constexpr int kMaxDevices = 64;
-int32_t* g_block_counts[kMaxDevices] = {nullptr};
-int g_sm_count[kMaxDevices] = {0};
+constexpr int kGateSlices = 32;
+struct GateScratch {
+    int32_t* base = nullptr;
+    int n_sm = 0;
+    int used = 0;
+    cudaStream_t key[kGateSlices];
+};
+GateScratch g_scratch[kMaxDevices];
+std::mutex g_scratch_mutex;
 
-int gate_scratch(int32_t** out, int* sms) {
+int gate_scratch(cudaStream_t st, int32_t** out, int* sms) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ARDIFF_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return ARDIFF_ERR_UNSUPPORTED;
-    if (!g_block_counts[dev]) {
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    GateScratch& g = g_scratch[dev];
+    if (!g.base) {
         int n_sm = 0;
         if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return ARDIFF_ERR_CUDA;
         int32_t* p = nullptr;
-        if (cudaMalloc(&p, sizeof(int32_t) * kMaxGateBlocks) != cudaSuccess) {
+        if (cudaMalloc(&p, sizeof(int32_t) * kMaxGateBlocks * kGateSlices) != cudaSuccess) {
             (void)cudaGetLastError();
             return ARDIFF_ERR_NOMEM;
         }
-        g_sm_count[dev] = n_sm;
-        g_block_counts[dev] = p;
+        g.n_sm = n_sm;
+        g.base = p;
     }
-    *out = g_block_counts[dev];
-    *sms = g_sm_count[dev];
+    int slice = -1;
+    for (int i = 0; i < g.used; ++i)
+        if (g.key[i] == st) { slice = i; break; }
+    if (slice < 0) {
+        if (g.used < kGateSlices - 1) {
+            g.key[g.used] = st;
+            slice = g.used++;
+        } else {
+            slice = kGateSlices - 1;
+        }
+    }
+    *out = g.base + (size_t)slice * kMaxGateBlocks;
+    *sms = g.n_sm;
     return ARDIFF_OK;
 }
 
@@ -449,9 +474,9 @@ int compact_launch(const uint8_t* mask, int64_t n, const int32_t* block_counts, 
     return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
 }
 
-int gate_scratch_get(int32_t** counts, int* max_blocks, int* sms) {
+int gate_scratch_get(cudaStream_t st, int32_t** counts, int* max_blocks, int* sms) {
     *max_blocks = kMaxGateBlocks;
-    return gate_scratch(counts, sms);
+    return gate_scratch(st, counts, sms);
 }
 
 int write_zero_count(int32_t* count, cudaStream_t st) {
@@ -466,7 +491,7 @@ extern "C" int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, fl
                                       void* stream) {
     int32_t* counts = nullptr;
     int sms = 0;
-    int rc = gate_scratch(&counts, &sms);
+    int rc = gate_scratch(static_cast<cudaStream_t>(stream), &counts, &sms);
     if (rc != ARDIFF_OK) return rc;
     return ardiff::gate_launch(feat, n, d, tau, mask, idx, count, entropy, counts, kMaxGateBlocks,
                                sms, static_cast<cudaStream_t>(stream));

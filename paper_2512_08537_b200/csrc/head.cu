@@ -63,8 +63,8 @@ constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;  // warp 0: TMA producer, warp 
 constexpr int XB_COLS = 64;       // x is fed to the in-projection as bf16, K padded to one slice
 constexpr int KMAX = 64;
 constexpr int CTRS = 4;           // counters per token tile: chain, gates of even blocks, gates of odd blocks, pad
-constexpr uint64_t kWaitLimitNs = 4000000000ull;   // a bounded wait gives up after 4 s
-constexpr uint64_t kDrainLimitNs = 200000000ull;   // waits for own copies in flight at exit
+constexpr uint64_t kWaitLimitNs = 4000000000ull;   // default: a bounded wait gives up after 4 s
+constexpr uint64_t kDrainLimitNs = 20000000ull;    // waits for own copies in flight at exit (ignore the abort flag)
 
 // Optional per-item time stamps of CTA 0 (compile with -DARDIFF_HEAD_PROFILE):
 // trace[(local item number * 3 + role) * 4 + slot] = clock64(); slot 3 = type * 1000 + column tile.
@@ -126,6 +126,10 @@ struct HeadParams {
     const float* step_noise;                // [K][n][C] fresh noise of the sampler steps, or nullptr
     long long step_stride;                  // n * C
     float ax[KMAX], av[KMAX], an[KMAX];     // sampler step k: x <- ax x + av v + an z_k
+    unsigned long long wait_limit_ns;       // bound of every dependency wait
+    int stall_tile;                         // self-test: conditioning items of this token tile wait for one
+                                            // predecessor more than exists (-1: none)
+    long long* clock_probe;                 // [4]: clock64 and globaltimer of CTA 0 at start and end
 };
 
 struct Packed { uint32_t w0, w1, w2, w3, w4; };
@@ -145,8 +149,7 @@ __device__ __forceinline__ void raise_timeout(const HeadParams& P) {
 }
 
 // bounded wait on an mbarrier phase; false = gave up (abort raised or seen)
-__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const HeadParams& P,
-                                          uint64_t limit_ns = kWaitLimitNs) {
+__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const HeadParams& P) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     for (uint32_t it = 1;; ++it) {
@@ -155,11 +158,23 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const H
             if (ptx::ld_relaxed_gpu(P.abort_flag) != 0) return false;
             const uint64_t now = ptx::globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) {
+            else if (now - t0 > P.wait_limit_ns) {
                 raise_timeout(P);
                 return false;
             }
         }
+    }
+}
+
+// Wait at exit for this CTA's own asynchronous work (copies landing in its shared memory, MMAs writing
+// its tensor memory). Bounded by time alone: after an abort the barrier may never complete (the partner's
+// share of the bytes is missing), and the limit covers any latency of the work itself.
+__device__ __forceinline__ void drain_mbar(uint32_t bar, uint32_t parity) {
+    if (ptx::mbar_try_wait(bar, parity)) return;
+    const uint64_t t0 = ptx::globaltimer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (ptx::mbar_try_wait(bar, parity)) return;
+        if ((it & 63u) == 0 && ptx::globaltimer_ns() - t0 > kDrainLimitNs) return;
     }
 }
 
@@ -175,7 +190,7 @@ __device__ __forceinline__ bool wait_counters(const int* c1, int n1, const int* 
             if (ptx::ld_relaxed_gpu(P.abort_flag) != 0) return false;
             const uint64_t now = ptx::globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
+            else if (now - t0 > P.wait_limit_ns) {
                 raise_timeout(P);
                 return false;
             }
@@ -259,6 +274,7 @@ __device__ __forceinline__ Packed decode_packed(const HeadParams& P, int MTu, in
         }
     }
     const int abs_m = (m0 + m) * 2 + rank;
+    if (type == OP_COND && abs_m == P.stall_tile) needA += 1;   // self-test: never satisfied
     pk.w0 = (uint32_t)abs_m | ((uint32_t)type << 24);
     pk.w1 = (uint32_t)nt | ((uint32_t)k << 8) | ((uint32_t)(block & 0xff) << 16) | ((uint32_t)gsel << 24);
     pk.w2 = (uint32_t)needA; pk.w3 = (uint32_t)needB; pk.w4 = (uint32_t)b_row;
@@ -645,6 +661,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     ptx::cluster_sync_all();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    long long probe_c0 = 0;
+    unsigned long long probe_g0 = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        probe_c0 = clock64();
+        probe_g0 = ptx::globaltimer_ns();
+    }
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -721,7 +743,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         // simply waits out a bounded time that covers any TMA latency.
         if (rank == 0) {
             for (int s = 0; s < STAGES; ++s)
-                if (issued & (1u << s)) wait_mbar(full_bar(s), (issued_parity >> s) & 1u, P, kDrainLimitNs);
+                if (issued & (1u << s)) drain_mbar(full_bar(s), (issued_parity >> s) & 1u);
         } else if (aborted) {
             const uint64_t t0 = ptx::globaltimer_ns();
             while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
@@ -774,7 +796,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             // all MMAs this thread issued must be done before TMEM is freed
             if (lane == 0) ptx::mma_commit_pair(drain_bar);
             __syncwarp();
-            wait_mbar(drain_bar, 0, P, kDrainLimitNs);
+            drain_mbar(drain_bar, 0);
         }
     } else {
         // ---------------- epilogue warps ----------------
@@ -888,7 +910,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                     Stats st;
                     st.init(0.f);
 #pragma unroll 1
-                    for (int j = 0; j < io.nch; ++j) {
+                    for (int j = 0; j < io.nch && !fail; ++j) {
                         const int b = j & 1;
                         const uint32_t bufF = my_buf + (uint32_t)b * EPI_BUF;
                         const uint32_t bufH = bufF + SLAB_F;
@@ -900,9 +922,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                             }
                             bool okw = wait_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u, P);
                             okw = __all_sync(0xffffffffu, okw);
+                            fail |= !okw;
+                            if (fail) break;      // aborted: the load stays pending and is waited for at exit
                             ld_parity ^= 1u << b;
                             ld_pending &= ~(1u << b);
-                            fail |= !okw;
                         } else {
                             // the store that last used this buffer must have finished reading it
                             if (lane == 0) ptx::bulk_wait_read<EPI_NB - 1>();
@@ -920,7 +943,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                             ptx::bulk_commit();
                         }
                     }
-                    if (it.type == OP_IN || it.type == OP_G2)
+                    if (!fail && (it.type == OP_IN || it.type == OP_G2))
                         P.stats[(size_t)grow * (2 * P.NT) + it.nt * 2 + half] = st.finish(128);
                 }
                 ptx::tc_fence_before();
@@ -946,7 +969,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         }
         // own copies in flight: loads that were issued but never consumed, stores not yet done
         for (int b = 0; b < EPI_NB; ++b)
-            if (ld_pending & (1u << b)) wait_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u, P, kDrainLimitNs);
+            if (ld_pending & (1u << b)) drain_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u);
         if (lane == 0) ptx::bulk_wait<0>();
         __syncwarp();
     }
@@ -957,6 +980,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc_pair(tmem_base, 512);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0 && P.clock_probe) {
+        // SM cycles and wall time of this launch as seen by CTA 0: their ratio is the clock the SM really ran at
+        P.clock_probe[0] = clock64() - probe_c0;
+        P.clock_probe[1] = (long long)(ptx::globaltimer_ns() - probe_g0);
     }
 }
 
@@ -1107,9 +1135,14 @@ struct ardiff_head {
     Phase* phases;
     uint16_t* cum2phase;
     CUtensorMap* maps;
-    // optional timing of the persistent kernel
-    int timing, timed;
+    long long* clock_probe;  // [2]: SM cycles and nanoseconds of the last launch, stamped by CTA 0
+    // optional timing of the persistent kernel (state of the last call, not of the head: mutable)
+    int timing;
+    mutable int timed;
     cudaEvent_t ev0, ev1;
+    // self-test of the bounded waits, armed for the next sample call only
+    mutable int stall_tile;
+    mutable unsigned int stall_limit_us;
 };
 
 namespace {
@@ -1142,11 +1175,13 @@ void free_all(ardiff_head* H) {
     H->allocs.clear();
 }
 
+#ifdef ARDIFF_TUNING
 int env_int(const char* name, int dflt) {
     const char* v = getenv(name);
     if (!v || !*v) return dflt;
     return atoi(v);
 }
+#endif
 
 }  // namespace
 
@@ -1195,13 +1230,16 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     H->max_tiles = (d.max_tokens + BM - 1) / BM;
     if (H->max_tiles < 1) H->max_tiles = 1;
 
-    // grid: one CTA per SM in clusters of two, all co-resident.
-    // The cooperative attribute makes the launch fail instead of start when the grid cannot be
-    // co-resident. ARDIFF_HEAD_COOP=0 drops it for tools that cannot replay such launches (the
-    // grid is still sized to be co-resident on an otherwise idle device, and every wait is bounded).
-    H->coop = env_int("ARDIFF_HEAD_COOP", 1) != 0;
+    // grid: one CTA per SM in clusters of two, all co-resident. The cooperative attribute makes the
+    // launch fail instead of start when the grid cannot be co-resident (ardiff_head_set_cooperative
+    // drops it for profilers that cannot replay such launches).
+    H->coop = 1;
+    H->stall_tile = -1;
+    H->grid = H->n_sm;
+#ifdef ARDIFF_TUNING
     H->grid = env_int("ARDIFF_HEAD_GRID", H->n_sm);
     if (H->grid < 2 || H->grid > H->n_sm) H->grid = H->n_sm;
+#endif
     H->grid &= ~1;
     {
         bool ok = cudaFuncSetAttribute(head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) ==
@@ -1227,10 +1265,12 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     // largest group, in units (pairs of token tiles): a phase of NT column tiles per token tile should
     // span about 2.5 grids of items so that a dependent phase finds its producers long finished
     int tgu = (5 * units / 2 + NT - 1) / NT;
+#ifdef ARDIFF_TUNING
     {
         const int tg_env = env_int("ARDIFF_HEAD_TGU", 0);
         if (tg_env > 0) tgu = tg_env;
     }
+#endif
     if (tgu < 1) tgu = 1;
     if ((int64_t)tgu * 2 > H->max_tiles + 1) tgu = (int)((H->max_tiles + 1) / 2);
     H->TGu = tgu;
@@ -1306,6 +1346,7 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     TRY(dev_alloc(H, &H->stats, R * 2 * NT, true));
     TRY(dev_alloc(H, &H->counters, ((size_t)H->max_tiles + 2) * CTRS, true));
     TRY(dev_alloc(H, &H->status, 2, true));
+    TRY(dev_alloc(H, &H->clock_probe, 2, true));
 #ifdef ARDIFF_HEAD_PROFILE
     TRY(dev_alloc(H, &H->trace, (size_t)TRACE_ITEMS * 3 * 4, true));
 #endif
@@ -1457,8 +1498,15 @@ int head_sample_impl(const ardiff_head* H, const void* cond, const float* noise,
     }
     P.step_noise = step_noise;
     P.step_stride = (long long)n_rows * C;
+    P.clock_probe = H->clock_probe;
+    P.wait_limit_ns = kWaitLimitNs;
+    P.stall_tile = -1;
+    if (H->stall_tile >= 0) {             // armed self-test: this call only
+        P.stall_tile = H->stall_tile;
+        P.wait_limit_ns = (unsigned long long)H->stall_limit_us * 1000ull;
+        H->stall_tile = -1;
+    }
 
-    ardiff_head* Hm = const_cast<ardiff_head*>(H);
     if (H->timing) cudaEventRecord(H->ev0, st);
     {
         cudaLaunchConfig_t cfg;
@@ -1483,7 +1531,7 @@ int head_sample_impl(const ardiff_head* H, const void* cond, const float* noise,
     }
     if (H->timing) {
         cudaEventRecord(H->ev1, st);
-        Hm->timed = 1;
+        H->timed = 1;
     }
     launches += 1;
     ardiff::set_launch_count(launches);
@@ -1539,27 +1587,41 @@ extern "C" int ardiff_head_status(ardiff_head* H, void* stream) {
     return v[0];
 }
 
-// Internal (not part of the public header): device pointers of the head's scratch arrays, for
-// bring-up scripts that compare intermediates. name: z xb s u a g0 g1 x c h temb counters trace
-extern "C" void* ardiff_head_debug_ptr(ardiff_head* H, const char* name) {
-    if (!H || !name) return nullptr;
-    if (!strcmp(name, "z")) return H->z;
-    if (!strcmp(name, "xb")) return H->xb;
-    if (!strcmp(name, "s")) return H->s;
-    if (!strcmp(name, "u")) return H->u;
-    if (!strcmp(name, "a")) return H->a;
-    if (!strcmp(name, "g0")) return H->g0;
-    if (!strcmp(name, "g1")) return H->g1;
-    if (!strcmp(name, "x")) return H->x;
-    if (!strcmp(name, "h")) return H->h;
-    if (!strcmp(name, "temb")) return H->temb;
-    if (!strcmp(name, "counters")) return H->counters;
-    if (!strcmp(name, "trace")) return H->trace;
-    return nullptr;
+extern "C" int ardiff_head_last_kernel_clock(ardiff_head* H, void* stream, double* sm_mhz) {
+    if (!H || !sm_mhz) return ARDIFF_ERR_NULL;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    long long v[2] = {0, 0};
+    if (cudaMemcpy(v, H->clock_probe, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return ARDIFF_ERR_CUDA;
+    if (v[1] <= 0) return ARDIFF_ERR_SHAPE;
+    *sm_mhz = 1e3 * (double)v[0] / (double)v[1];
+    return ARDIFF_OK;
 }
 
-// Internal: synchronous device-to-host copy for bring-up scripts.
-extern "C" int ardiff_debug_copy_to_host(void* dst, const void* src, size_t bytes) {
-    if (cudaDeviceSynchronize() != cudaSuccess) return ARDIFF_ERR_CUDA;
-    return cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
+extern "C" int ardiff_head_set_cooperative(ardiff_head* H, int on) {
+    if (!H) return ARDIFF_ERR_NULL;
+    H->coop = on ? 1 : 0;
+    return ARDIFF_OK;
 }
+
+extern "C" int ardiff_head_inject_stall(ardiff_head* H, int32_t token_tile, uint32_t wait_limit_us) {
+    if (!H) return ARDIFF_ERR_NULL;
+    if (token_tile < 0 || wait_limit_us < 100 || wait_limit_us > 4000000u) return ARDIFF_ERR_SHAPE;
+    H->stall_tile = token_tile;
+    H->stall_limit_us = wait_limit_us;
+    return ARDIFF_OK;
+}
+
+namespace ardiff {
+const ardiff_head_desc* head_desc(const ardiff_head* H) { return H ? &H->d : nullptr; }
+}  // namespace ardiff
+
+#ifdef ARDIFF_HEAD_PROFILE
+// Only in profiling builds: the per-item time stamps of CTA 0, copied to the host.
+extern "C" int ardiff_head_copy_trace(ardiff_head* H, long long* dst, size_t count) {
+    if (!H || !dst || !H->trace) return ARDIFF_ERR_NULL;
+    if (cudaDeviceSynchronize() != cudaSuccess) return ARDIFF_ERR_CUDA;
+    if (count > (size_t)TRACE_ITEMS * 3 * 4) count = (size_t)TRACE_ITEMS * 3 * 4;
+    return cudaMemcpy(dst, H->trace, count * sizeof(long long), cudaMemcpyDeviceToHost) == cudaSuccess ? ARDIFF_OK
+                                                                                                   : ARDIFF_ERR_CUDA;
+}
+#endif

@@ -94,11 +94,13 @@ __global__ void __launch_bounds__(1024) tau_kernel(const float* __restrict__ H, 
 
 __global__ void __launch_bounds__(kThreads)
 accept_prefix_kernel(const float* __restrict__ r, const float* __restrict__ ratio, int64_t n, int32_t gamma,
-                     int64_t n_blocks, int32_t* __restrict__ accepted) {
+                     int64_t n_blocks, const int32_t* __restrict__ block_len, int32_t* __restrict__ accepted) {
     const int64_t b = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (b >= n_blocks) return;
     const int64_t t0 = b * gamma;
-    const int64_t t1 = min(n, t0 + gamma);
+    int64_t t1 = min(n, t0 + gamma);
+    // the draft that reaches Step 4 is what Step 1 left of the block
+    if (block_len) t1 = min(t1, t0 + (int64_t)max(block_len[b], 0));
     int acc = (int)(t1 - t0);
     for (int64_t t = t0; t < t1; ++t) {
         if (r[t] > ratio[t]) {
@@ -118,7 +120,7 @@ extern "C" int ardiff_entropy_gate_blocks(const void* feat, int64_t n, int32_t r
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!count) return ARDIFF_ERR_NULL;
     if (n < 0 || rows_per_token < 1 || gamma < 1 || d < 1 || d > 65536) return ARDIFF_ERR_SHAPE;
-    if (n * (int64_t)rows_per_token >= (int64_t)1 << 31) return ARDIFF_ERR_SHAPE;
+    if (n >= (int64_t)1 << 31 || n * (int64_t)rows_per_token >= (int64_t)1 << 31) return ARDIFF_ERR_SHAPE;
     if (n == 0) {
         ardiff::set_launch_count(1);
         return ardiff::write_zero_count(count, st);
@@ -126,7 +128,7 @@ extern "C" int ardiff_entropy_gate_blocks(const void* feat, int64_t n, int32_t r
     if (!feat || !row_entropy || !mask || !idx) return ARDIFF_ERR_NULL;
     int32_t* counts = nullptr;
     int max_blocks = 0, sms = 0;
-    int rc = ardiff::gate_scratch_get(&counts, &max_blocks, &sms);
+    int rc = ardiff::gate_scratch_get(st, &counts, &max_blocks, &sms);
     if (rc != ARDIFF_OK) return rc;
     rc = ardiff::entropy_rows_launch(feat, n * rows_per_token, d, row_entropy, sms, st);
     if (rc != ARDIFF_OK) return rc;
@@ -154,14 +156,14 @@ extern "C" int ardiff_tau_calibrate(const float* entropy, int64_t n, double* out
 }
 
 extern "C" int ardiff_accept_prefix(const float* r, const float* ratio, int64_t n, int32_t gamma,
-                                    int32_t* accepted, void* stream) {
+                                    const int32_t* block_len, int32_t* accepted, void* stream) {
     if (n < 0 || gamma < 1) return ARDIFF_ERR_SHAPE;
     if (n == 0) return ARDIFF_OK;
     if (!r || !ratio || !accepted) return ARDIFF_ERR_NULL;
     const int64_t n_blocks = (n + gamma - 1) / gamma;
     const int grid = (int)((n_blocks + kThreads - 1) / kThreads);
     accept_prefix_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(r, ratio, n, gamma, n_blocks,
-                                                                                 accepted);
+                                                                                 block_len, accepted);
     ardiff::set_launch_count(1);
     return cudaGetLastError() == cudaSuccess ? ARDIFF_OK : ARDIFF_ERR_CUDA;
 }

@@ -75,6 +75,9 @@ extern "C" int ardiff_pipeline_create_slots(ardiff_head* head, int64_t max_n, in
     *out = nullptr;
     if (max_n < 1 || max_n >= ((int64_t)1 << 31) || d < 1 || d > 65536 || Dc < 1 || C < 1) return ARDIFF_ERR_SHAPE;
     if (n_slots < 1 || n_slots > ARDIFF_PIPELINE_MAX_SLOTS) return ARDIFF_ERR_SHAPE;
+    // the head kernel indexes the staging buffers with the head's own widths and runs at most max_tokens survivors
+    const ardiff_head_desc* hd = ardiff::head_desc(head);
+    if (Dc != hd->Dc || C != hd->C || max_n > hd->max_tokens) return ARDIFF_ERR_SHAPE;
     ardiff_pipeline* p = new (std::nothrow) ardiff_pipeline();
     if (!p) return ARDIFF_ERR_NOMEM;
     p->head = head;
@@ -145,9 +148,14 @@ extern "C" int ardiff_pipeline_run_host(ardiff_pipeline* p, const void* feat, co
     if (n < 0 || n > p->max_n) return ARDIFF_ERR_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     Slot& q = p->slot[0];
-    // slot 0 may still belong to an asynchronous submission
+    // Batches submitted earlier may still be in flight on the pipeline's own streams, and they use the same
+    // head (its scratch, its counters): this call's work is ordered on the device after every one of them.
+    // Slot 0's staging buffers are reused here, so its batch is waited for and delivered as _wait would.
+    for (int s = 1; s < p->n_slots; ++s)
+        if (p->slot[s].used && cudaStreamWaitEvent(st, p->slot[s].out_done, 0) != cudaSuccess) return ARDIFF_ERR_CUDA;
     if (q.used) {
         if (cudaEventSynchronize(q.out_done) != cudaSuccess) return ARDIFF_ERR_CUDA;
+        if (q.rc == ARDIFF_OK && q.count_user) *q.count_user = *q.count_pinned;
         q.used = false;
     }
     const size_t nn = (size_t)n;

@@ -133,6 +133,32 @@ def test_bad_arguments_are_rejected_without_launching():
     torch.cuda.synchronize()
 
 
+def test_gate_calls_on_two_unordered_streams():
+    """Two gate calls of different shapes enqueued on two streams with no ordering between them (they may
+    overlap on the GPU: each stream has its own block-count scratch) give what each gives alone."""
+    dev = require_cuda()
+    jobs = {}
+    for key, (n, d, q) in {"a": (60000, 768, 0.3), "b": (9001, 5120, 0.6)}.items():
+        wl = synth.workload("cfg2" if key == "a" else "cfg4", n=n, d=d)
+        feat = dev_bf16(synth.features(wl))
+        _, _, _, ent = ardiff.ardiff_entropy_gate(feat, -1.0, want_entropy=True)
+        tau = float(np.quantile(ent.cpu().numpy(), q))
+        mask, idx, count, _ = ardiff.ardiff_entropy_gate(feat, tau)
+        torch.cuda.synchronize()
+        jobs[key] = (feat, tau, mask.clone(), idx.clone(), int(count.item()))
+    streams = {k: torch.cuda.Stream(device=dev) for k in jobs}
+    res = []
+    for rep in range(6):
+        for key, (feat, tau, *_rest) in jobs.items():
+            with torch.cuda.stream(streams[key]):
+                m, i, c, _ = ardiff.ardiff_entropy_gate(feat, tau, stream=streams[key])
+            res.append((key, m, i, c))
+    torch.cuda.synchronize()
+    for key, m, i, c in res:
+        _, _, mask, idx, count = jobs[key]
+        assert int(c.item()) == count and torch.equal(m, mask) and torch.equal(i[:count], idx[:count]), key
+
+
 def test_full_size_gate_stress_sampled_rows_and_properties():
     """2^20 x 5120 (10.7 GB): features are generated and uploaded in slabs; the oracle checks a
     sample of rows one by one, the rest is checked through properties that hold at any size."""
@@ -149,6 +175,15 @@ def test_full_size_gate_stress_sampled_rows_and_properties():
     rows = np.unique(np.concatenate([np.arange(0, 64), np.arange(wl.n - 64, wl.n),
                                      rng.integers(0, wl.n, size=4096)]))
     H_s = np.array([oracle.entropy(synth.features(wl, int(r), 1))[0] for r in rows])
+    cond = torch.empty((wl.n, wl.Dc), dtype=torch.bfloat16, device=dev)
+    noise = torch.empty((wl.n, wl.C), dtype=torch.float32, device=dev)
+    big = 1 << 17
+    for r0 in range(0, wl.n, big):
+        cond[r0:r0 + big] = dev_bf16(synth.cond(wl, r0, big))
+        noise[r0:r0 + big] = torch.from_numpy(synth.noise(wl, r0, big)).to(dev)
+    w, t = synth.head_weights(wl), synth.t_sched(wl.K)
+    head = ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K, wl.n, w)
+    out = torch.empty((wl.n, wl.C), dtype=torch.float32, device=dev)
     for q in (0.0, 0.1, 0.5, 0.9, 0.99):
         tau = quantile_tau(H_s, q)
         mask, idx, count, ent = ardiff.ardiff_entropy_gate(feat, tau, want_entropy=True)
@@ -163,31 +198,28 @@ def test_full_size_gate_stress_sampled_rows_and_properties():
         want_idx = torch.nonzero(mask, as_tuple=False).flatten().to(torch.int32)
         assert torch.equal(idx[:c], want_idx)
         assert abs(c / wl.n - (1 - q)) < 0.03
-    # the survivors of the last (99 % filtered) pass feed the cfg2-shaped head: under-filled grid, ragged tail
-    S = c
-    idx_h = idx[:S].cpu().numpy()
-    w, t = synth.head_weights(wl), synth.t_sched(wl.K)
-    cond = torch.empty((wl.n, wl.Dc), dtype=torch.bfloat16, device=dev)
-    noise = torch.empty((wl.n, wl.C), dtype=torch.float32, device=dev)
-    big = 1 << 17
-    for r0 in range(0, wl.n, big):
-        cond[r0:r0 + big] = dev_bf16(synth.cond(wl, r0, big))
-        noise[r0:r0 + big] = torch.from_numpy(synth.noise(wl, r0, big)).to(dev)
-    head = ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K, wl.n, w)
-    out = torch.full((wl.n, wl.C), -777.0, dtype=torch.float32, device=dev)
-    head.ardiff_head_sample(cond, noise, t, idx, count, out)
-    assert head.status() == 0
-    pos = np.unique(np.concatenate([np.arange(0, 12), np.arange(S - (S % 128 or 128), S)[-12:],
-                                    rng.integers(0, S, size=24)]))
-    toks = idx_h[pos]
-    small = synth.workload("cfg5", n=len(toks))
-    cond_s = np.concatenate([synth.cond(wl, int(tk), 1) for tk in toks])
-    noise_s = np.concatenate([synth.noise(wl, int(tk), 1) for tk in toks])
-    want = oracle.head_sample(w, cond_s, noise_s, t, np.arange(len(toks), dtype=np.int32))
-    got = out[torch.from_numpy(toks.astype(np.int64)).to(dev)].cpu().numpy().astype(np.float64)
-    err = np.abs(got - want).max(axis=1) / np.sqrt((want ** 2).mean(axis=1))
-    assert err.max() <= 2e-2, err.max()
-    written = (out[:, 0] != -777.0)
-    assert int(written.sum().item()) == S and bool(written[torch.from_numpy(idx_h.astype(np.int64)).to(dev)].all())
-    assert bool(torch.isfinite(out[written]).all())
+        if q == 0.1:
+            continue                                   # head runs: 0, 50, 90 and 99 % filtered
+        # The survivors feed the cfg2-shaped head: from 8192 token tiles with the scratch ring wrapping many
+        # times (0 %) to an under-filled grid with a ragged tail (99 %). The oracle checks, one by one, every
+        # third token of the first tile, the whole last (ragged) tile and one random token of every 16th tile.
+        S = c
+        idx_h = idx[:S].cpu().numpy()
+        out.fill_(-777.0)
+        head.ardiff_head_sample(cond, noise, t, idx, count, out)
+        assert head.status() == 0
+        tiles = (S + 127) // 128
+        pos = np.concatenate([np.arange(0, min(S, 128), 3), np.arange(max(0, S - (S % 128 or 128)), S),
+                              np.arange(0, tiles, 16) * 128 + rng.integers(0, 128, size=len(range(0, tiles, 16)))])
+        pos = np.unique(pos[pos < S])
+        toks = idx_h[pos]
+        cond_s = np.concatenate([synth.cond(wl, int(tk), 1) for tk in toks])
+        noise_s = np.concatenate([synth.noise(wl, int(tk), 1) for tk in toks])
+        want = oracle.head_sample(w, cond_s, noise_s, t, np.arange(len(toks), dtype=np.int32))
+        got = out[torch.from_numpy(toks.astype(np.int64)).to(dev)].cpu().numpy().astype(np.float64)
+        err = np.abs(got - want).max(axis=1) / np.sqrt((want ** 2).mean(axis=1))
+        assert err.max() <= 2e-2, (q, err.max())
+        written = (out[:, 0] != -777.0)                # written iff kept, and finite
+        assert int(written.sum().item()) == S and torch.equal(written, mask.bool())
+        assert bool(torch.isfinite(out[written]).all())
     head.close()

@@ -2,16 +2,20 @@
 
 Agreement bar: per token, max |out - oracle| <= 2e-2 * RMS(oracle row) (bf16 GEMM operands, fp32
 accumulation on the GPU; no rounding in the oracle). The same bar is applied to the velocity
-(out - noise) on one-step runs, where the noise no longer props up the RMS.
+(out - noise) on one-step runs, where the noise no longer props up the RMS. On the full-size
+workloads, where several hundred tokens are compared, a token that misses the bar is looked up in
+the CPU rounding model (gpu_util.assert_head_parity): it may pass only if bf16 rounding alone
+already puts it there.
 """
 import numpy as np
 import pytest
 import torch
 
 import oracle
+import rounding_model
 import synth
 import paper_2512_08537_b200 as ardiff
-from gpu_util import dev_bf16, dev_f32, require_cuda
+from gpu_util import assert_head_parity, dev_bf16, dev_f32, require_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -184,9 +188,9 @@ def test_full_size_runs_are_bit_identical(name, runs, K):
 @pytest.mark.parametrize("name,extra,K", [("cfg2", 160, None), ("cfg3", 48, None), ("cfg4", 32, None),
                                           ("cfg3", 24, 1), ("cfg3", 12, 8)])
 def test_workload_configs_sampled_tokens(name, extra, K):
-    """Full-size gate -> head run; the oracle checks the first, a middle and the last (ragged)
-    token tile plus random survivors one by one (tokens are independent). cfg 3 also runs at the
-    other step counts its workload names (K = 1 and 8)."""
+    """Full-size gate -> head run; the oracle checks one token of every token tile, the first, a middle
+    and the last (ragged) token tile and random survivors one by one (tokens are independent). cfg 3
+    also runs at the other step counts its workload names (K = 1 and 8)."""
     dev = require_cuda()
     wl = synth.workload(name) if K is None else synth.workload(name, K=K)
     feat_bits = synth.features(wl)
@@ -203,17 +207,25 @@ def test_workload_configs_sampled_tokens(name, extra, K):
     S = int(count.item())
     idx_h = idx.cpu().numpy()[:S]
     got = out.cpu().numpy()
-    if name != "cfg2":                      # keep the oracle's share of the run to seconds
-        pos = sample_tokens(idx_h, extra=extra)
-        edge = 16 if K is None else 6
-        pos = np.concatenate([pos[:edge], pos[len(pos) // 2: len(pos) // 2 + edge // 2], pos[-edge:],
-                              np.random.default_rng(1).choice(pos, size=extra, replace=False)])
-        pos = np.unique(pos)
-    else:
-        pos = sample_tokens(idx_h, extra=extra)
+    # Oracle-checked, element by element: one random token of EVERY token tile (an error confined to some
+    # tiles, a group boundary or a scratch-slot reuse cannot hide), plus the whole first, one middle and the
+    # last (ragged) tile and some random survivors. At the other step counts of cfg 3 the whole tiles are
+    # thinned to keep the oracle's share of the run to seconds.
+    rng = np.random.default_rng(11)
+    tiles = (S + 127) // 128
+    per_tile = np.minimum(np.arange(tiles) * 128 + rng.integers(0, 128, size=tiles), S - 1)
+    whole = sample_tokens(idx_h, extra=extra)
+    if K is not None:
+        whole = whole[::4]
+    pos = np.unique(np.concatenate([per_tile, whole]))
     toks = idx_h[pos]
     want = oracle.head_sample(w, cond_bits, noise, t, toks)
-    assert_parity(got, want, toks, name)
+
+    def floor(rows):        # what bf16 rounding alone costs these tokens (CPU model, fp64)
+        exact = rounding_model.head(w, cond_bits, noise, t, rows, rounded=())
+        return rounding_model.error_ratio(rounding_model.head(w, cond_bits, noise, t, rows), exact)
+
+    assert_head_parity(got, want, toks, name, model=floor)
     # properties that hold for every token: written iff kept, finite
     kept = np.zeros(wl.n, bool)
     kept[idx_h] = True
@@ -287,10 +299,8 @@ def test_linear_sampler_steps(sampler):
     """Other samplers on the same head: every step is x <- ax x + av v + an z_k."""
     dev = require_cuda()
     wl = synth.workload("cfg1", n=300, K=4)
-    # Euler and eps-prediction keep the state (ax != 0) and run on the harder 1/sqrt(fan_in) weights; the
-    # x0-prediction sampler returns the head's raw last output after two compounding passes and runs on
-    # the workloads' own weight recipe, N(0, 0.02)
-    w = synth.head_weights(wl, std=0.02 if sampler == "x0_renoise" else None)
+    # all three on the harder 1/sqrt(fan_in) weights (every layer keeps unit scale, nothing damps an error)
+    w = synth.head_weights(wl, std=None)
     cond_bits, noise = synth.cond(wl), synth.noise(wl)
     idx_np = np.random.default_rng(7).permutation(wl.n)[:211].astype(np.int32)
     z = None
@@ -340,4 +350,32 @@ def test_extreme_shapes(shape):
     head = make_head(wl, w)
     got = run_head(head, cond_bits, noise, t, idx)
     assert_parity(got, want, idx, str(shape))
+    head.close()
+
+
+def test_bounded_wait_runs_out_reports_timeout_and_the_head_recovers():
+    """The self-test hook makes one tile's dependency wait unsatisfiable and shortens the wait limit to 3 ms:
+    the kernel must come back by itself (no fault, no trap, no endless spin), the status word must say
+    TIMEOUT, and the very next call on the same head must give the bits of an undisturbed run."""
+    wl = synth.workload("cfg1", n=900)
+    w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    idx = np.arange(wl.n, dtype=np.int32)
+    head = make_head(wl, w)
+    clean = run_head(head, cond_bits, noise, t, idx)
+    for tile in (0, 3, 7):                                # first, an odd (partner CTA) and the last, ragged tile
+        head.inject_stall(tile, 3000)
+        dev = require_cuda()
+        out = torch.zeros(noise.shape, dtype=torch.float32, device=dev)
+        head.ardiff_head_sample(dev_bf16(cond_bits), dev_f32(noise), t, torch.from_numpy(idx).to(dev),
+                                torch.tensor([wl.n], dtype=torch.int32, device=dev), out)
+        assert head.status() == ardiff.ARDIFF_ERR_TIMEOUT
+        assert head.status() == 0                         # reading the status clears it
+        assert np.array_equal(run_head(head, cond_bits, noise, t, idx), clean)
+    head.inject_stall(4000, 3000)                         # a tile this call does not have: no effect
+    assert np.array_equal(run_head(head, cond_bits, noise, t, idx), clean)
+    fresh = make_head(wl, w)
+    assert np.array_equal(run_head(fresh, cond_bits, noise, t, idx), clean)
+    with pytest.raises(ardiff.ArdiffError):
+        head.inject_stall(0, 5)                           # limit below 100 us
+    fresh.close()
     head.close()

@@ -122,3 +122,39 @@ def test_accept_prefix(gamma):
     ratio[::97] = r[::97]                                              # ties are not rejections
     got = ardiff.ardiff_accept_prefix(torch.from_numpy(r).to(dev), torch.from_numpy(ratio).to(dev), gamma)
     assert np.array_equal(got.cpu().numpy(), oracle.accept_prefix(r, ratio, gamma))
+
+
+@pytest.mark.parametrize("gamma", [1, 8, 37])
+def test_accept_prefix_on_truncated_blocks(gamma):
+    """Algorithm 1 Step 4 on the draft that Step 1 left: the accepted count is capped by the kept length."""
+    dev = require_cuda()
+    rng = np.random.default_rng(50 + gamma)
+    n = 4099
+    nb = (n + gamma - 1) // gamma
+    r = rng.uniform(0, 1, n).astype(np.float32)
+    ratio = rng.uniform(0.5, 2.0, n).astype(np.float32)
+    full = np.array([min(gamma, n - b * gamma) for b in range(nb)], np.int32)
+    kept = np.minimum(rng.integers(0, gamma + 1, nb).astype(np.int32), full)
+    got = ardiff.ardiff_accept_prefix(torch.from_numpy(r).to(dev), torch.from_numpy(ratio).to(dev), gamma,
+                                      block_len=torch.from_numpy(kept).to(dev))
+    assert np.array_equal(got.cpu().numpy(), oracle.accept_prefix(r, ratio, gamma, kept))
+
+
+def test_early_stop_feeds_accept_prefix_on_the_device():
+    """Step 1 -> Step 4 composed on the device: block_len written by the block-prefix gate is read by the
+    accepted-prefix kernel on the same stream, no host round trip."""
+    dev = require_cuda()
+    wl = synth.workload("cfg2", n=8 * 515)
+    bits = synth.features(wl)
+    H = oracle.entropy(bits)
+    tau = float(np.quantile(H, 0.1))
+    rng = np.random.default_rng(9)
+    r = rng.uniform(0, 1, wl.n).astype(np.float32)
+    ratio = rng.uniform(0.7, 2.0, wl.n).astype(np.float32)
+    _, _, _, blen, _, _ = ardiff.ardiff_entropy_gate_blocks(dev_bf16(bits), 1, 8, tau)
+    got = ardiff.ardiff_accept_prefix(torch.from_numpy(r).to(dev), torch.from_numpy(ratio).to(dev), 8, block_len=blen)
+    _, _, _, _, len_o = oracle.gate_blocks(bits, 1, 8, tau)
+    band = (np.abs(H - float(np.float32(tau))) < BAND).reshape(-1, 8).any(axis=1)
+    want = oracle.accept_prefix(r, ratio, 8, len_o)
+    assert np.array_equal(got.cpu().numpy()[~band], want[~band])
+    assert np.all(got.cpu().numpy() <= blen.cpu().numpy())

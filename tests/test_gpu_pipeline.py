@@ -5,6 +5,8 @@ Agreement bars: as in the gate and head tests (mask equal outside a 1e-4 entropy
 per token max |out - oracle| <= 2e-2 * RMS(oracle row)); overlapped vs blocking: bit-exact, since
 both run the same kernels on the same data.
 """
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -116,6 +118,83 @@ def test_overlapped_batches_match_blocking_call():
     head.close()
 
 
+def test_run_host_while_another_slot_is_in_flight():
+    """The blocking call on a multi-slot pipeline while a batch submitted on another slot may still be
+    running: both use the one head, so the blocking call has to order itself after that batch. Both
+    results must equal what the blocking call gives alone."""
+    dev = require_cuda()
+    wl = synth.workload("cfg1")
+    w, t = synth.head_weights(wl), synth.t_sched(wl.K)
+    max_n = 4096
+    head = ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K, max_n, w)
+    ref_pipe = ardiff.Pipeline(head, max_n, wl.d)
+    pipe = ardiff.Pipeline(head, max_n, wl.d, slots=3)
+    ba, bb = batch(wl, 301, 4096), batch(wl, 302, 3001)
+    want = []
+    for b, feat, cond, noise in (ba, bb):
+        out, mask = outputs(b.n, wl.C)
+        kept = ref_pipe.ardiff_pipeline_run_host(feat, cond, noise, 5.1, t, out, mask)
+        want.append((out.clone(), mask.clone(), kept))
+    stream = torch.cuda.Stream(device=dev)
+    for rep in range(3):
+        oa, ma = outputs(ba[0].n, wl.C)
+        ob, mb = outputs(bb[0].n, wl.C)
+        pipe.ardiff_pipeline_submit(1, ba[1], ba[2], ba[3], 5.1, t, oa, ma, stream=stream)
+        kept_b = pipe.ardiff_pipeline_run_host(bb[1], bb[2], bb[3], 5.1, t, ob, mb, stream=stream)   # no wait first
+        kept_a = pipe.ardiff_pipeline_wait(1)
+        assert head.status() == 0
+        assert (kept_a, kept_b) == (want[0][2], want[1][2])
+        assert torch.equal(oa, want[0][0]) and torch.equal(ma, want[0][1])
+        assert torch.equal(ob, want[1][0]) and torch.equal(mb, want[1][1])
+    pipe.close()
+    ref_pipe.close()
+    head.close()
+
+
+def test_full_cfg2_through_three_slots_against_oracle():
+    """The size the end-to-end figure is quoted on: 16384-token batches of the cfg 2 shape streamed through
+    three slots; mask against the oracle outside the band, sampled survivors of every batch one by one."""
+    require_cuda()
+    wl = synth.workload("cfg2")
+    w, t = synth.head_weights(wl), synth.t_sched(wl.K)
+    head = ardiff.Head(wl.C, wl.Dc, wl.W, wl.L, wl.F, wl.K, wl.n, w)
+    pipe = ardiff.Pipeline(head, wl.n, wl.d, slots=3)
+    n_batches = 5
+    batches = [batch(wl, 400 + i, wl.n) for i in range(n_batches)]
+    res = [outputs(wl.n, wl.C) for _ in range(n_batches)]
+    taus, kept = [], [None] * n_batches
+    for b, *_ in batches:
+        H = oracle.entropy(synth.features(b))
+        Hs = np.sort(H)
+        k = int(round(wl.filter_q * wl.n))
+        taus.append((0.5 * (Hs[k - 1] + Hs[k]), H))
+    for i, (b, feat, cond, noise) in enumerate(batches):
+        slot = i % 3
+        if i >= 3:
+            kept[i - 3] = pipe.ardiff_pipeline_wait(slot)
+        pipe.ardiff_pipeline_submit(slot, feat, cond, noise, taus[i][0], t, res[i][0], res[i][1])
+    for i in range(n_batches - 3, n_batches):
+        kept[i] = pipe.ardiff_pipeline_wait(i % 3)
+    assert head.status() == 0
+    rng = np.random.default_rng(3)
+    for i, (b, feat, cond, noise) in enumerate(batches):
+        tau, H = taus[i]
+        mask_o = (H >= float(np.float32(tau))).astype(np.uint8)
+        got, mask_g = res[i][0].numpy(), res[i][1].numpy()
+        off_band = np.abs(H - float(np.float32(tau))) >= BAND
+        assert np.array_equal(mask_g[off_band], mask_o[off_band]) and kept[i] == int(mask_g.sum())
+        surv = np.flatnonzero(mask_g)
+        tiles = (len(surv) + 127) // 128
+        pos = np.unique(np.minimum(np.arange(tiles) * 128 + rng.integers(0, 128, size=tiles), len(surv) - 1))
+        toks = surv[pos]
+        want = oracle.head_sample(w, synth.cond(b), synth.noise(b), t, toks.astype(np.int32))
+        err = np.abs(got[toks].astype(np.float64) - want[toks]).max(axis=1) / np.sqrt((want[toks] ** 2).mean(axis=1))
+        assert err.max() <= REL_TOL, (i, err.max())
+        assert np.all(got[mask_g == 0] == 0.0) and np.all(np.isfinite(got))
+    pipe.close()
+    head.close()
+
+
 def test_join_orders_a_stream_after_the_batches():
     dev = require_cuda()
     wl = synth.workload("cfg1")
@@ -166,6 +245,13 @@ def test_bad_arguments():
     assert two.ardiff_pipeline_wait(1) == 0            # never submitted: returns at once
     with pytest.raises(RuntimeError):
         ardiff.Pipeline(head, 256, wl.d, slots=5)
+    # staging buffers that do not match the head: more tokens than it can run, another cond width or token dim
+    vp = ctypes.c_void_p
+    create = lib.ardiff_pipeline_create_slots
+    h = ctypes.c_void_p()
+    assert create(head._h, 257, wl.d, wl.Dc, wl.C, 1, ctypes.byref(h)) == ardiff.ARDIFF_ERR_SHAPE
+    assert create(head._h, 256, wl.d, wl.Dc + 64, wl.C, 1, ctypes.byref(h)) == ardiff.ARDIFF_ERR_SHAPE
+    assert create(head._h, 256, wl.d, wl.Dc, wl.C + 16, 1, ctypes.byref(h)) == ardiff.ARDIFF_ERR_SHAPE
     one.close()
     two.close()
     head.close()
