@@ -310,6 +310,58 @@ def run_sweep(torch, ardiff, dev, pk, flush, stream, main_wl, main_batch, main_h
     return recs
 
 
+def run_next_stage(torch, ardiff, dev, pk, flush, stream):
+    """Timings of the later-stage entry points (block-prefix gate, threshold statistics, accepted prefix)
+    beside the plain gate on the same input: median of 15 calls, L2 flushed before each."""
+    recs = []
+
+    def timed(fn, reps=15):
+        ts = []
+        for i in range(reps + 3):
+            flush.fill_(i & 0xff)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            e1.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    def rec(call, shape, ms, nbytes):
+        recs.append({"call": call, "shape": shape, "us": ms * 1e3, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                     "frac_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"]})
+
+    wl = synth.workload("cfg2")
+    feat = upload_bf16(torch, synth.features(wl), dev)
+    n, d = feat.shape
+    mask = torch.empty(n, dtype=torch.uint8, device=dev)
+    idx = torch.empty(n, dtype=torch.int32, device=dev)
+    count = torch.zeros(1, dtype=torch.int32, device=dev)
+    ent = torch.empty(n, dtype=torch.float32, device=dev)
+    ardiff.ardiff_entropy_gate(feat, -1.0, mask, idx, count, ent)
+    torch.cuda.synchronize()
+    tau = quantile_tau(ent.cpu().numpy().astype(np.float64), 0.05)
+    by = n * (2 * d + 5) + 4
+    shape = f"{n} tokens x {d}"
+    rec("ardiff_entropy_gate", shape, timed(lambda: ardiff.ardiff_entropy_gate(feat, tau, mask, idx, count)), by)
+    rec("ardiff_entropy_gate_blocks gamma=8", shape,
+        timed(lambda: ardiff.ardiff_entropy_gate_blocks(feat, 1, 8, tau, want_row_entropy=False)), by + n // 8 * 4)
+    rec("ardiff_entropy_gate_stats", shape, timed(lambda: ardiff.ardiff_entropy_gate_stats(feat, tau)), by + 24)
+    rec("ardiff_tau_calibrate", f"{n} entropies", timed(lambda: ardiff.ardiff_tau_calibrate(ent)), 4 * n + 24)
+    r_ = torch.rand(n, device=dev)
+    ratio = torch.rand(n, device=dev) + 0.5
+    rec("ardiff_accept_prefix gamma=8", f"{n} tokens", timed(lambda: ardiff.ardiff_accept_prefix(r_, ratio, 8)),
+        8 * n + n // 8 * 4)
+    # attention-map-shaped input: 16 rows (heads x query rows) of 1024 keys per token
+    wl2 = synth.workload("cfg3", n=4096 * 16)
+    feat2 = upload_bf16(torch, synth.features(wl2), dev)
+    rec("ardiff_entropy_gate_blocks rows_per_token=16 gamma=8", "4096 tokens x 16 rows x 1024",
+        timed(lambda: ardiff.ardiff_entropy_gate_blocks(feat2, 16, 8, 6.0, want_row_entropy=False)),
+        feat2.numel() * 2 + 4096 * 5)
+    return recs
+
+
 def run_gpu(args, wl):
     import torch
     import paper_2512_08537_b200 as ardiff
@@ -532,6 +584,7 @@ def run_gpu(args, wl):
         }
         if world == 1 and not args.no_sweep:
             line["sweep"] = run_sweep(torch, ardiff, dev, pk, flush, stream, wl, b, head, log)
+            line["next_stage"] = run_next_stage(torch, ardiff, dev, pk, flush, stream)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl, weights, args.cpu_tokens, args.cpu_tokens_one_core)
         print(json.dumps(line), flush=True)

@@ -74,6 +74,17 @@ int ardiff_entropy_gate(const void* feat, int64_t n, int32_t d, float tau, uint8
 int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask,
                            int32_t* idx, int32_t* count, float* entropy, void* stream);
 
+/* The gate together with the statistics that the paper's threshold equation needs ("Entropy-Based
+ * Early Stopping in Inference Phase": tau_ent = 0.3 E[H] - 0.1 std(H)), in the same pass over the
+ * features: the row kernel leaves per-block partial sums (fp64) beside its counts and the compaction
+ * kernel merges them in a fixed order. Run it on a calibration batch with any tau (e.g. -1: keep all)
+ * and use out3[2] as the threshold of the following calls.
+ *   out3  dev double [3]  out: { mean(H), std(H) with divisor n, 0.3 mean - 0.1 std } over the n rows
+ *         (a row with NaN entropy makes all three NaN). Reproducible run to run for a given n and d.
+ *   entropy  as in the _ex form, may be NULL.  n >= 1.  Everything else as ardiff_entropy_gate. */
+int ardiff_entropy_gate_stats(const void* feat, int64_t n, int32_t d, float tau, uint8_t* mask,
+                              int32_t* idx, int32_t* count, float* entropy, double* out3, void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * Block-prefix gate: the early stop as the paper's Algorithm 1, Step 1 writes it ("if H^s <
  * tau_ent: draft_tokens <- draft_tokens[1 : i-1]; break"). Tokens come in draft blocks of
@@ -84,7 +95,10 @@ int ardiff_entropy_gate_ex(const void* feat, int64_t n, int32_t d, float tau, ui
  * token with indicator < tau (or NaN) drops itself and every later token of the block.
  *
  *   feat           dev bf16 [n * rows_per_token][d], alignment as for ardiff_entropy_gate
- *   row_entropy    dev float [n * rows_per_token]  out (also the kernels' scratch), required
+ *   row_entropy    dev float [n * rows_per_token]  out, or NULL. One pass over the features does all of it
+ *                  (row entropies stay in shared memory) when d % 8 == 0, d <= 8192 and
+ *                  gamma * rows_per_token <= 24576; other shapes go through row_entropy as scratch and
+ *                  return ARDIFF_ERR_NULL without it
  *   token_entropy  dev float [n]  out, or NULL
  *   mask, idx, count   as for ardiff_entropy_gate (idx ascending)
  *   block_len      dev int32 [ceil(n / gamma)]  out, or NULL: tokens kept in each block

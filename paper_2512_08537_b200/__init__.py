@@ -129,6 +129,27 @@ def ardiff_entropy_gate(feat, tau: float, mask=None, idx=None, count=None, entro
     return mask, idx, count, entropy
 
 
+def ardiff_entropy_gate_stats(feat, tau: float = -1.0, want_entropy: bool = False, stream=None):
+    """Gate + threshold statistics of its own entropies in one pass. Returns (mask, idx, count, entropy or
+    None, out3 float64 CUDA tensor [3] = mean, std, 0.3 mean - 0.1 std)."""
+    import torch
+    assert feat.is_cuda and feat.dtype == torch.bfloat16 and feat.dim() == 2 and feat.is_contiguous()
+    n, d = feat.shape
+    dev = feat.device
+    mask = torch.empty((n,), dtype=torch.uint8, device=dev)
+    idx = torch.empty((max(n, 1),), dtype=torch.int32, device=dev)
+    count = torch.empty((1,), dtype=torch.int32, device=dev)
+    entropy = torch.empty((n,), dtype=torch.float32, device=dev) if want_entropy else None
+    out3 = torch.empty((3,), dtype=torch.float64, device=dev)
+    vp = ctypes.c_void_p
+    fn = _fn("ardiff_entropy_gate_stats", [vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, vp, vp, vp, vp, vp, vp])
+    with torch.cuda.device(dev):
+        rc = fn(feat.data_ptr(), n, d, float(tau), mask.data_ptr(), idx.data_ptr(), count.data_ptr(),
+                entropy.data_ptr() if entropy is not None else None, out3.data_ptr(), _stream_ptr(stream))
+    _check(rc, "ardiff_entropy_gate_stats")
+    return mask, idx, count, entropy, out3
+
+
 def _fn(name, argtypes):
     """A library function with its ctypes signature set (lazily, once)."""
     fn = getattr(lib(), name)
@@ -139,7 +160,7 @@ def _fn(name, argtypes):
 
 
 def ardiff_entropy_gate_blocks(feat, rows_per_token: int, gamma: int, tau: float, want_token_entropy: bool = False,
-                               stream=None):
+                               want_row_entropy: bool = True, stream=None):
     """Block-prefix gate (early stop inside draft blocks of `gamma` tokens, each token owning
     `rows_per_token` rows of feat). Returns (mask u8 [n], idx i32 [n], count i32 [1], block_len i32
     [ceil(n/gamma)], row_entropy f32 [n*rows_per_token], token_entropy f32 [n] or None)."""
@@ -156,10 +177,11 @@ def ardiff_entropy_gate_blocks(feat, rows_per_token: int, gamma: int, tau: float
     idx = torch.empty((max(n, 1),), dtype=torch.int32, device=dev)
     count = torch.empty((1,), dtype=torch.int32, device=dev)
     block_len = torch.empty((max((n + gamma - 1) // gamma, 1),), dtype=torch.int32, device=dev)
-    row_ent = torch.empty((max(rows, 1),), dtype=torch.float32, device=dev)
+    row_ent = torch.empty((max(rows, 1),), dtype=torch.float32, device=dev) if want_row_entropy else None
     tok_ent = torch.empty((max(n, 1),), dtype=torch.float32, device=dev) if want_token_entropy else None
     with torch.cuda.device(dev):
-        rc = fn(feat.data_ptr(), n, rows_per_token, d, gamma, float(tau), row_ent.data_ptr(),
+        rc = fn(feat.data_ptr(), n, rows_per_token, d, gamma, float(tau),
+                row_ent.data_ptr() if row_ent is not None else None,
                 tok_ent.data_ptr() if tok_ent is not None else None, mask.data_ptr(), idx.data_ptr(),
                 count.data_ptr(), block_len.data_ptr(), _stream_ptr(stream))
     _check(rc, "ardiff_entropy_gate_blocks")

@@ -66,6 +66,6 @@ extern "C" int ardiff_entropy_gate_noalloc(const void* feat, int64_t n, int32_t 
     int sms = 0;
     const int rc = static_scratch(&counts, &sms);
     if (rc != ARDIFF_OK) return rc;
-    return ardiff::gate_launch(feat, n, d, tau, mask, idx, count, nullptr, counts, kStaticGateBlocks, sms,
-                               static_cast<cudaStream_t>(stream));
+    return ardiff::gate_launch(feat, n, d, tau, mask, idx, count, nullptr, counts, nullptr, nullptr,
+                               kStaticGateBlocks, sms, static_cast<cudaStream_t>(stream));
 }

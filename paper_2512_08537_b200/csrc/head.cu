@@ -6,23 +6,25 @@
 //
 // How: every matrix product of the head is cut into items of 128 tokens x 256 output columns. The two
 // CTAs of a cluster form a unit: each owns one token tile, stages its own A tile (activations) and
-// half of the B tile (weights) per 64-wide K slice by TMA into a 4-stage shared-memory ring, and the
+// half of the B tile (weights) per 64-wide K slice by TMA into a 6-stage shared-memory ring, and the
 // even CTA issues tcgen05.mma.cta_group::2 (256 x 256 x 16, bf16 -> fp32) into one of two TMEM
 // accumulators. Eight epilogue warps per CTA read the accumulator back with tcgen05.ld and apply the
 // fused tail of the layer (bias, SiLU, LayerNorm statistics, LayerNorm + modulation, gated residual,
-// Euler update, scatter) while the next item's MMAs run; their global operands and results move as
-// swizzled 32 x 32 slabs by TMA.
+// Euler update, scatter) while the next item's MMAs run. Results that a later GEMM reads as an operand
+// (s, u, a) leave as swizzled bf16 slabs by TMA stores; the residual stream h and the gate values, which
+// only epilogues touch, move between registers and global memory directly in a layout made for that.
 // All items of a call form one static list (a per-step "program" of phases, repeated for every step
 // and every group of token tiles); unit u takes items u, u + units, ... . The modulation GEMM of a
 // block is split: its gate third does not depend on the residual stream, so gate items of block b+1
 // are placed between the dependent phases of block b, where they cover the latency of the chain.
 // Dependencies between items are tracked per token tile by three counters (chain, gates of even
 // blocks, gates of odd blocks) with release/acquire at gpu scope; every wait is bounded.
-// The binding resource is the SM's shared-memory bandwidth (about 128 B/clk): at tensor peak the operand
-// ring alone takes all of it (32 KB written by TMA and 32 KB read by the MMA per 512-cycle stage), and every
-// byte an epilogue stages in a slab is paid twice. Hence biases travel in registers (one column per lane,
-// handed round by shuffle), c never leaves the accumulator, and proxy fences sit only where a proxy is
-// really crossed: a fence in the producer's path stalls the whole ring.
+// What binds it: the rate at which operand tiles reach shared memory. Without cluster multicast every CTA
+// pulls its own 32 KB per 64-wide K slice out of L2 (62 B/clk at tensor peak); a slice is in flight for
+// 2-4 thousand cycles and the copies complete at 50-55 B/clk per SM however many are outstanding. So the
+// kernel keeps everything else off that path and off the producer's instruction stream: biases travel in
+// registers (one column per lane, handed round by shuffle), c never leaves the accumulator, epilogue inputs
+// are plain loads issued three units ahead, and proxy fences sit only where a proxy is really crossed.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -46,18 +48,18 @@ constexpr int BN = 256;           // output columns per item (UMMA N)
 constexpr int BK = 64;            // K slice per pipeline stage (128 bytes of bf16: one swizzle row)
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_ROWS = BN / 2;    // rows of the weight tile that one CTA of the pair stages
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int STAGE_BYTES = A_BYTES + B_ROWS * BK * 2;   // 32 KB
-// epilogue staging: every epilogue warp owns EPI_NB buffers, each one fp32 slab (32 rows x 128 B,
-// 128-byte swizzle) plus one bf16 slab (32 rows x 64 B, 64-byte swizzle), filled and drained by TMA
+// epilogue staging: every epilogue warp owns EPI_NB bf16 slabs (32 rows x 64 B, 64-byte swizzle) for the
+// results that later GEMMs read as operands (s, u, a): written by the lanes, drained by TMA stores.
+// Everything else an epilogue reads or writes (h, gate values, x) moves between registers and global memory
+// directly, so that shared memory belongs to the operand ring: its depth, not its bandwidth, sets the pace.
 constexpr int EPI_WARPS = 8;
 constexpr int EPI_NB = 2;
-constexpr int SLAB_F = 32 * 128;
 constexpr int SLAB_H = 32 * 64;
-constexpr int EPI_BUF = SLAB_F + SLAB_H;
-constexpr int EPI_BYTES = EPI_WARPS * EPI_NB * EPI_BUF;
+constexpr int EPI_BYTES = EPI_WARPS * EPI_NB * SLAB_H;
 constexpr int DEP_BARS = 8;       // the producer runs at most 6 items ahead of the epilogue
-constexpr int NUM_BARS = 2 * STAGES + 5 + DEP_BARS + EPI_WARPS * EPI_NB;
+constexpr int NUM_BARS = 2 * STAGES + 5 + DEP_BARS;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*align slack*/ + 8 * NUM_BARS + 16;
 constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
 constexpr int XB_COLS = 64;       // x is fed to the in-projection as bf16, K padded to one slice
@@ -71,10 +73,16 @@ constexpr uint64_t kDrainLimitNs = 20000000ull;    // waits for own copies in fl
 #ifdef ARDIFF_HEAD_PROFILE
 constexpr int TRACE_ITEMS = 4096;
 #define TRACE(role, slot) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + (slot)] = clock64(); } while (0)
-#define TRACE_TYPE(role) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + 3] = it.type * 1000 + it.nt; } while (0)
-#define TRACE_DECL int trace_n = 0;
+#define TRACE_TYPE(role) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + 3] = it.type * 1000 + it.nt + ((role) == 0 ? 100 * trace_flag : 0); } while (0)
+#define TRACE_DECL int trace_n = 0; int trace_flag = 0;
+#define TRACE_FLAG(x) trace_flag = (x)
 #define TRACE_NEXT() ++trace_n
+// per pipeline stage of the first 16 K slices of an item: role 0 = load issued, role 1 = MMA saw the stage full
+// (bit 0 of the stamp: it had to wait for it)
+#define TRACE_STAGE(role, kb) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS / 2 && (kb) < 16) P.trace[(size_t)TRACE_ITEMS * 12 + ((size_t)trace_n * 16 + (kb)) * 2 + (role)] = clock64(); } while (0)
 #else
+#define TRACE_STAGE(role, kb)
+#define TRACE_FLAG(x)
 #define TRACE(role, slot)
 #define TRACE_TYPE(role)
 #define TRACE_DECL
@@ -84,7 +92,7 @@ constexpr int TRACE_ITEMS = 4096;
 enum OpType : int { OP_GATHER = 0, OP_COND, OP_IN, OP_SS, OP_GATE, OP_G1, OP_G2, OP_FSS, OP_OUT, OP_NOP, OP_END = 15 };
 enum MapId : int {
     MAP_Z = 0, MAP_XB, MAP_S, MAP_U, MAP_A, MAP_WC, MAP_WIN, MAP_WCAT, MAP_WOUT,   // GEMM operands
-    EMAP_H, EMAP_S, EMAP_U, EMAP_A, EMAP_G0, EMAP_G1,                       // epilogue slabs
+    EMAP_S, EMAP_U, EMAP_A,                                                 // epilogue output slabs
     MAP_COUNT
 };
 
@@ -330,11 +338,14 @@ struct ItemStream {
 
 // ------------------------------------------------------------------------------------------
 // epilogues. Two epilogue warps share each 32-row quarter of the tile (TMEM lane quarter*32 + lane);
-// warp half h of the pair takes accumulator columns [128 h, 128 h + 128). Work goes in chunks of 32
-// accumulator columns: the chunk's global inputs (h, c: fp32 slab; g: bf16 slab) arrive by TMA in a
-// swizzled shared-memory buffer, the lane reads its own row, combines it with the accumulator chunk,
-// writes the results back into the buffer (in place) and lane 0 hands the buffer to a TMA store.
-// Loads run one chunk ahead.
+// warp half h of the pair takes accumulator columns [128 h, 128 h + 128). A thread owns one row and
+// works through it in units of 16 accumulator columns.
+//   h (fp32 residual stream) and the gate values (bf16) are read and written only by epilogue threads.
+//   They live in a layout of their own: chunks of 32 rows x 32 columns in which the 16-byte pieces of
+//   the 32 rows lie side by side, so that every 128-bit access of a warp is one contiguous 512 bytes.
+//   Loads go straight to registers (L2 only: other CTAs rewrite the data) and are issued three units
+//   ahead, the first ones before the accumulator is even complete.
+//   s, u, a are operands of later GEMMs (read by TMA): bf16 slabs in shared memory, drained by TMA stores.
 // ------------------------------------------------------------------------------------------
 struct Stats {
     float p, sd, sq;
@@ -348,84 +359,84 @@ struct Stats {
     }
 };
 
-struct EpiIO {            // what one warp moves per 32-column chunk of one item (-1: nothing)
-    int nch;              // chunks of this warp
-    int acc0;             // accumulator column of the warp's first chunk
-    int col0;             // global column of the warp's first chunk (slabs, biases)
-    int ldF, ldH, stF, stH;   // map ids
-};
-
-__device__ __forceinline__ EpiIO epi_io(const Item& it, int half) {
-    EpiIO io{4, half * 128, it.nt * BN + half * 128, -1, -1, -1, -1};
-    switch (it.type) {
-        case OP_COND: break;          // own path: one bf16 slab per step
-        case OP_IN: io.stF = EMAP_H; break;
-        case OP_SS:
-        case OP_FSS:
-            io.nch = 2; io.acc0 = half * 64; io.col0 = it.nt * 128 + half * 64;
-            io.ldF = EMAP_H; io.stH = EMAP_U;
-            break;
-        case OP_GATE: io.stH = EMAP_G0 + (it.gsel - 1); break;
-        case OP_G1: io.stH = EMAP_A; break;
-        case OP_G2: io.ldF = EMAP_H; io.ldH = EMAP_G0 + (it.gsel - 1); io.stF = EMAP_H; break;
-        default: io.nch = 0; break;   // OP_OUT: register path
-    }
-    return io;
-}
-
-__device__ __forceinline__ uint32_t slabF_addr(uint32_t base, int r, int c16) {
-    return base + r * 128 + ((c16 ^ (r & 7)) << 4);
-}
 __device__ __forceinline__ uint32_t slabH_addr(uint32_t base, int r, int c16) {
     return base + r * 64 + ((c16 ^ ((r >> 1) & 3)) << 4);
 }
 
-__device__ __forceinline__ void load_acc32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
-    ptx::tmem_ld_32x32b_x32(taddr, r);
+__device__ __forceinline__ void load_acc16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    ptx::tmem_ld_32x32b_x16(taddr, r);
     ptx::tmem_ld_wait();
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// The chunk's 32 bias values sit one per lane (fetched at the start of the item, while the accumulator is still
-// being produced) and are handed round by shuffle: no global load on the chunk's critical path.
-__device__ __forceinline__ void add_bias32(float (&v)[32], float b_lane) {
+// The 32 bias values of a 32-column chunk sit one per lane (fetched at the start of the item, while the
+// accumulator is still being produced) and are handed round by shuffle: no global load on the critical path.
+__device__ __forceinline__ void add_bias16(float (&v)[16], float b_lane, int lane0) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] += __shfl_sync(0xffffffffu, b_lane, i);
+    for (int i = 0; i < 16; ++i) v[i] += __shfl_sync(0xffffffffu, b_lane, lane0 + i);
 }
 
-__device__ __forceinline__ void slabF_read(uint32_t base, int r, float (&v)[32]) {
+// 16 columns of this lane's row as bf16 into a slab (pieces 2 hu and 2 hu + 1 of the row's four)
+__device__ __forceinline__ void slabH_write16(uint32_t base, int r, int hu, const float (&v)[16]) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        const uint4 w = ptx::lds_u4(slabF_addr(base, r, c));
-        v[4 * c] = __uint_as_float(w.x); v[4 * c + 1] = __uint_as_float(w.y);
-        v[4 * c + 2] = __uint_as_float(w.z); v[4 * c + 3] = __uint_as_float(w.w);
-    }
-}
-__device__ __forceinline__ void slabF_write(uint32_t base, int r, const float (&v)[32]) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c)
-        ptx::sts_u4(slabF_addr(base, r, c), make_uint4(__float_as_uint(v[4 * c]), __float_as_uint(v[4 * c + 1]),
-                                                       __float_as_uint(v[4 * c + 2]), __float_as_uint(v[4 * c + 3])));
-}
-__device__ __forceinline__ void slabH_read(uint32_t base, int r, float (&v)[32]) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const uint4 w = ptx::lds_u4(slabH_addr(base, r, c));
-        v[8 * c] = bf16lo(w.x); v[8 * c + 1] = bf16hi(w.x); v[8 * c + 2] = bf16lo(w.y); v[8 * c + 3] = bf16hi(w.y);
-        v[8 * c + 4] = bf16lo(w.z); v[8 * c + 5] = bf16hi(w.z); v[8 * c + 6] = bf16lo(w.w); v[8 * c + 7] = bf16hi(w.w);
-    }
-}
-__device__ __forceinline__ void slabH_write(uint32_t base, int r, const float (&v)[32]) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
         uint4 w;
         w.x = pack_bf16x2(v[8 * c], v[8 * c + 1]);
         w.y = pack_bf16x2(v[8 * c + 2], v[8 * c + 3]);
         w.z = pack_bf16x2(v[8 * c + 4], v[8 * c + 5]);
         w.w = pack_bf16x2(v[8 * c + 6], v[8 * c + 7]);
-        ptx::sts_u4(slabH_addr(base, r, c), w);
+        ptx::sts_u4(slabH_addr(base, r, 2 * hu + c), w);
+    }
+}
+
+// Chunked layout of h (fp32) and of the gate values (bf16): element (row, col) of a [rows][W] array lives
+// in chunk (row / 32, col / 32); inside the chunk the 16-byte piece p of the row's 32 columns of lane
+// row % 32 sits at 16-byte index p * 32 + lane. A 16-column unit u of a warp's span is pieces
+// 4 (u & 1) .. + 3 (fp32) or 2 (u & 1), + 1 (bf16) of chunk (first chunk + u / 2).
+__device__ __forceinline__ size_t chunk_of(const HeadParams& P, int row0, int col0) {
+    return (size_t)(row0 >> 5) * (size_t)(P.W >> 5) + (size_t)(col0 >> 5);
+}
+struct UnitH { float4 p[4]; };      // 16 fp32 of one row
+struct UnitG { uint4 p[2]; };       // 16 bf16 of one row
+__device__ __forceinline__ void load_unit_h(const float* h, size_t chunk, int u, int lane, UnitH& d) {
+    const float* src = h + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 4) * 128 + lane * 4;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) d.p[q] = ptx::ldcg_f4(src + q * 128);
+}
+__device__ __forceinline__ void store_unit_h(float* h, size_t chunk, int u, int lane, const float (&v)[16]) {
+    float* dst = h + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 4) * 128 + lane * 4;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) ptx::st_f4(dst + q * 128, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
+}
+__device__ __forceinline__ void load_unit_g(const bf16* g, size_t chunk, int u, int lane, UnitG& d) {
+    const bf16* src = g + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 2) * 256 + lane * 8;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) d.p[q] = ptx::ldcg_u4(src + q * 256);
+}
+__device__ __forceinline__ void store_unit_g(bf16* g, size_t chunk, int u, int lane, const float (&v)[16]) {
+    bf16* dst = g + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 2) * 256 + lane * 8;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        uint4 w;
+        w.x = pack_bf16x2(v[8 * q], v[8 * q + 1]);
+        w.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+        w.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+        w.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+        ptx::st_u4(dst + q * 256, w);
+    }
+}
+__device__ __forceinline__ void unit_h_values(const UnitH& d, float (&v)[16]) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { v[4 * q] = d.p[q].x; v[4 * q + 1] = d.p[q].y; v[4 * q + 2] = d.p[q].z; v[4 * q + 3] = d.p[q].w; }
+}
+__device__ __forceinline__ void unit_g_values(const UnitG& d, float (&v)[16]) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const uint4 w = d.p[q];
+        v[8 * q] = bf16lo(w.x); v[8 * q + 1] = bf16hi(w.x); v[8 * q + 2] = bf16lo(w.y); v[8 * q + 3] = bf16hi(w.y);
+        v[8 * q + 4] = bf16lo(w.z); v[8 * q + 5] = bf16hi(w.z); v[8 * q + 6] = bf16lo(w.w); v[8 * q + 7] = bf16hi(w.w);
     }
 }
 
@@ -447,66 +458,6 @@ __device__ __forceinline__ void row_mean_rstd(const HeadParams& P, int grow, flo
     mean = v0.x + dmean;
     m2 = fmaxf(m2 - (float)P.W * dmean * dmean, 0.f);
     rstd = rsqrtf(m2 / (float)P.W + 1e-6f);
-}
-
-// One 32-column chunk of one item. acc: TMEM address of the chunk; col: its global column (bias index
-// for the 256-column ops), bufF / bufH: this warp's slabs for the chunk; r: lane.
-__device__ __forceinline__ void epi_chunk(const HeadParams& P, const Item& it, uint32_t acc, int acc_col, int col,
-                                          bool first, uint32_t bufF, uint32_t bufH, int r, Stats& st, float mean,
-                                          float rstd, float b0, float b1) {
-    float v[32];
-    switch (it.type) {
-        case OP_IN: {                         // h = acc + bin
-            load_acc32(acc, v);
-            add_bias32(v, b0);
-            if (first) st.init(v[0]);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) st.add(v[i]);
-            slabF_write(bufF, r, v);
-            break;
-        }
-        case OP_SS:
-        case OP_FSS: {                        // u = LN(h) * (1 + scale) + shift
-            float sc[32], hv[32];
-            load_acc32(acc, v);
-            load_acc32(acc + 128, sc);
-            add_bias32(v, b0);
-            add_bias32(sc, b1);
-            slabF_read(bufF, r, hv);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], v[i]);
-            slabH_write(bufH, r, hv);
-            break;
-        }
-        case OP_GATE: {                       // g = acc + bias
-            load_acc32(acc, v);
-            add_bias32(v, b0);
-            slabH_write(bufH, r, v);
-            break;
-        }
-        case OP_G1: {                         // a = SiLU(acc + b1)
-            load_acc32(acc, v);
-            add_bias32(v, b0);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = silu_f(v[i]);
-            slabH_write(bufH, r, v);
-            break;
-        }
-        default: {                            // OP_G2: h += g * (acc + b2)
-            float gv[32], hv[32];
-            load_acc32(acc, v);
-            add_bias32(v, b0);
-            slabH_read(bufH, r, gv);
-            slabF_read(bufF, r, hv);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) hv[i] = fmaf(gv[i], v[i], hv[i]);
-            if (first) st.init(hv[0]);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) st.add(hv[i]);
-            slabF_write(bufF, r, hv);
-            break;
-        }
-    }
 }
 
 // v = acc + bout ; x <- ax_k x + av_k v + an_k z_k ; bf16 copy for the next in-projection ; last step: out[idx[j]] = x
@@ -617,9 +568,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
     auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
     const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
     auto dep_bar = [&](uint32_t i) { return bars + 8u * (2 * STAGES + 5 + (i % DEP_BARS)); };
-    auto epi_bar = [&](int w, int b) { return bars + 8u * (2 * STAGES + 5 + DEP_BARS + w * EPI_NB + b); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + EPI_BYTES + 8 * NUM_BARS);
-
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int rank = (int)ptx::cluster_ctarank();                  // token tile of the unit this CTA owns
@@ -649,8 +598,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         }
         ptx::mbar_init(drain_bar, 1);
         for (int i = 0; i < DEP_BARS; ++i) ptx::mbar_init(dep_bar(i), 1);
-        for (int w = 0; w < EPI_WARPS; ++w)
-            for (int b = 0; b < EPI_NB; ++b) ptx::mbar_init(epi_bar(w, b), 1);
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -713,6 +660,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (kb == 0) TRACE(0, 1);
+                TRACE_STAGE(0, kb);
                 if (lane == 0) {
                     const uint32_t sa = smem_base + stage * STAGE_BYTES;
                     // the even CTA arms its barrier for the bytes of both CTAs
@@ -772,6 +720,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                     ok = wait_mbar(full_bar(stage), phase, P);
                     ok = __all_sync(0xffffffffu, ok);
                     if (kb == 0) TRACE(1, 1);
+                    TRACE_STAGE(1, kb);
                     if (!ok) break;
                     ptx::tc_fence_after();
                     if (lane == 0) {
@@ -804,9 +753,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
         const int half = ew >> 2;             // column half of the accumulator this warp takes
         const int row = quarter * 32 + lane;  // row of the tile owned by this thread
-        const uint32_t my_buf = epi_base + (uint32_t)ew * EPI_NB * EPI_BUF;
-        uint32_t ld_parity = 0;               // bit b: parity to wait for on this warp's barrier b
-        uint32_t ld_pending = 0;              // bit b: a load into buffer b is in flight
+        const uint32_t my_buf = epi_base + (uint32_t)ew * EPI_NB * SLAB_H;
         uint32_t acc_iter = 0;
         uint32_t seq = 0;
         ItemStream ist;
@@ -831,38 +778,42 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 ++seq;
                 if (!ok) break;
                 if (ew == 0) TRACE(2, 0);
-                const EpiIO io = epi_io(it, half);
-                const bool has_loads = (io.ldF >= 0) || (io.ldH >= 0);
-                // h and the gate values were written by TMA stores and are read by TMA loads: no proxy is crossed
+                const bool mod = (it.type == OP_SS || it.type == OP_FSS);
+                // this warp's span: 128 accumulator columns (64 of shift and 64 of scale for a modulation item)
+                const int acc0 = mod ? half * 64 : half * 128;
+                const int col0 = mod ? it.nt * 128 + half * 64 : it.nt * BN + half * 128;   // column of the layer's output
                 const int row0 = it.slot_row0 + quarter * 32;
-                auto issue_load = [&](int j) {
-                    const int b = j & 1;
-                    if (lane == 0) {
-                        const uint32_t bar = epi_bar(ew, b);
-                        const uint32_t dst = my_buf + (uint32_t)b * EPI_BUF;
-                        ptx::mbar_arrive_expect_tx(bar, (io.ldF >= 0 ? SLAB_F : 0) + (io.ldH >= 0 ? SLAB_H : 0));
-                        if (io.ldF >= 0) ptx::tma_load_2d(dst, P.maps + io.ldF, bar, io.col0 + 32 * j, row0);
-                        if (io.ldH >= 0) ptx::tma_load_2d(dst + SLAB_F, P.maps + io.ldH, bar, io.col0 + 32 * j, row0);
+                const int grow = it.slot_row0 + row;
+                const size_t chunk0 = chunk_of(P, row0, col0);
+                // inputs that do not come from the accumulator are asked for now, three units deep, while the
+                // MMAs of this item still run
+                UnitH hin[4];
+                UnitG gin[4];
+                const bf16* gsrc = it.gsel == 2 ? P.g1 : P.g0;
+                if (it.type == OP_G2) {
+#pragma unroll
+                    for (int u = 0; u < 3; ++u) {
+                        load_unit_h(P.h, chunk0, u, lane, hin[u]);
+                        load_unit_g(gsrc, chunk0, u, lane, gin[u]);
                     }
-                    ld_pending |= 1u << b;
-                };
-                if (has_loads && io.nch > 0) issue_load(0);
+                } else if (mod) {
+#pragma unroll
+                    for (int u = 0; u < 3; ++u) load_unit_h(P.h, chunk0, u, lane, hin[u]);
+                }
                 // bias values of the warp's chunks, one column per lane (modulation items: shift in bq[0..1], scale in bq[2..3])
                 float bq[4] = {0.f, 0.f, 0.f, 0.f};
                 {
-                    const bool mod = (it.type == OP_SS || it.type == OP_FSS);
-                    const float* bb = it.type == OP_IN     ? P.bin + io.col0
-                                      : it.type == OP_COND ? P.bc + io.col0
-                                                           : P.bias_cat + it.b_row + io.acc0;
+                    const float* bb = it.type == OP_IN     ? P.bin + col0
+                                      : it.type == OP_COND ? P.bc + col0
+                                                           : P.bias_cat + it.b_row + acc0;
                     if (it.type != OP_OUT) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             bq[q] = __ldg(bb + (mod ? (q & 1) * 32 + (q >> 1) * 128 : q * 32) + lane);
                     }
                 }
-                const int grow = it.slot_row0 + row;
                 float mean = 0.f, rstd = 0.f;
-                if (it.type == OP_SS || it.type == OP_FSS) row_mean_rstd(P, grow, mean, rstd);
+                if (mod) row_mean_rstd(P, grow, mean, rstd);
                 const uint32_t buf = acc_iter & 1u;
                 const uint32_t acc_phase = (acc_iter >> 1) & 1u;
                 ok = wait_mbar(tfull_bar(buf), acc_phase, P);
@@ -871,86 +822,145 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 if (ew == 0) TRACE(2, 1);
                 ptx::tc_fence_after();
                 const uint32_t tacc = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
-                if (it.type == OP_OUT) {
-                    if (!fail && half == 0) epi_out(P, it, tacc, grow, it.abs_m * BM + row, count);
-                } else if (it.type == OP_COND) {
-                    // c = acc + bc stays in registers; s_k = SiLU(c + temb_k) leaves as one bf16 slab per step.
-                    // The warp's shared memory holds six such slabs; a slab is reused three stores later.
-                    if (lane == 0) ptx::bulk_wait_read<0>();
+                // a slab may be rewritten once the TMA store that read it last (two stores back) is done reading
+                auto slab_ready = [&]() {
+                    if (lane == 0) ptx::bulk_wait_read<EPI_NB - 1>();
                     __syncwarp();
+                };
+                auto slab_store = [&](int map, uint32_t slab, int col, int grow0) {
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(P.maps + map, slab, col, grow0);
+                        ptx::bulk_commit();
+                    }
+                };
+                if (fail) {
+                    // aborted: nothing valid to work on
+                } else if (it.type == OP_OUT) {
+                    if (half == 0) epi_out(P, it, tacc, grow, it.abs_m * BM + row, count);
+                } else if (it.type == OP_COND) {
+                    // c = acc + bc stays in registers; s_k = SiLU(c + temb_k) leaves as one bf16 slab per step
                     int n_st = 0;
 #pragma unroll 1
-                    for (int j = 0; j < io.nch && !fail; ++j) {
+                    for (int j = 0; j < 4; ++j) {
                         float cv[32];
-                        load_acc32(tacc + io.acc0 + 32 * j, cv);
-                        add_bias32(cv, j == 0 ? bq[0] : j == 1 ? bq[1] : j == 2 ? bq[2] : bq[3]);
-                        float tk = __ldg(P.temb + io.col0 + 32 * j + lane);          // temb_k of this lane's column
+                        {
+                            float lo[16], hi[16];
+                            load_acc16(tacc + acc0 + 32 * j, lo);
+                            load_acc16(tacc + acc0 + 32 * j + 16, hi);
+                            const float bj = j == 0 ? bq[0] : j == 1 ? bq[1] : j == 2 ? bq[2] : bq[3];
+                            add_bias16(lo, bj, 0);
+                            add_bias16(hi, bj, 16);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) { cv[i] = lo[i]; cv[16 + i] = hi[i]; }
+                        }
+                        float tk = __ldg(P.temb + col0 + 32 * j + lane);          // temb_k of this lane's column
 #pragma unroll 1
                         for (int k = 0; k < P.K; ++k, ++n_st) {
                             const float tcur = tk;
-                            if (k + 1 < P.K) tk = __ldg(P.temb + (size_t)(k + 1) * P.W + io.col0 + 32 * j + lane);
-                            const uint32_t sl = my_buf + (uint32_t)(n_st % 6) * SLAB_H;
-                            if (n_st >= 6) {
-                                if (lane == 0) ptx::bulk_wait_read<5>();
-                                __syncwarp();
-                            }
-                            float sv[32];
+                            if (k + 1 < P.K) tk = __ldg(P.temb + (size_t)(k + 1) * P.W + col0 + 32 * j + lane);
+                            const uint32_t sl = my_buf + (uint32_t)(n_st & 1) * SLAB_H;
+                            slab_ready();
+                            float sv[16];
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) sv[i] = silu_f(cv[i] + __shfl_sync(0xffffffffu, tcur, i));
-                            slabH_write(sl, lane, sv);
-                            ptx::fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == 0) {
-                                ptx::tma_store_2d(P.maps + EMAP_S, sl, io.col0 + 32 * j, k * P.R + row0);
-                                ptx::bulk_commit();
+                            for (int hu = 0; hu < 2; ++hu) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    sv[i] = silu_f(cv[16 * hu + i] + __shfl_sync(0xffffffffu, tcur, 16 * hu + i));
+                                slabH_write16(sl, lane, hu, sv);
                             }
+                            slab_store(EMAP_S, sl, col0 + 32 * j, k * P.R + row0);
                         }
+                    }
+                } else if (it.type == OP_IN) {
+                    // h = acc + bin, straight to global memory; LayerNorm partials of the 128 columns
+                    Stats st;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        float v[16];
+                        load_acc16(tacc + acc0 + 16 * u, v);
+                        add_bias16(v, (u >> 1) == 0 ? bq[0] : (u >> 1) == 1 ? bq[1] : (u >> 1) == 2 ? bq[2] : bq[3], 16 * (u & 1));
+                        if (u == 0) st.init(v[0]);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) st.add(v[i]);
+                        store_unit_h(P.h, chunk0, u, lane, v);
+                    }
+                    P.stats[(size_t)grow * (2 * P.NT) + it.nt * 2 + half] = st.finish(128);
+                } else if (it.type == OP_GATE) {
+                    // g = acc + bias, as bf16 straight to global memory
+                    bf16* gdst = it.gsel == 2 ? P.g1 : P.g0;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        float v[16];
+                        load_acc16(tacc + acc0 + 16 * u, v);
+                        add_bias16(v, (u >> 1) == 0 ? bq[0] : (u >> 1) == 1 ? bq[1] : (u >> 1) == 2 ? bq[2] : bq[3], 16 * (u & 1));
+                        store_unit_g(gdst, chunk0, u, lane, v);
+                    }
+                } else if (it.type == OP_G1) {
+                    // a = SiLU(acc + b1): operand of the next GEMM, leaves as bf16 slabs
+#pragma unroll 1
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t sl = my_buf + (uint32_t)(j & 1) * SLAB_H;
+                        const float bj = j == 0 ? bq[0] : j == 1 ? bq[1] : j == 2 ? bq[2] : bq[3];
+                        slab_ready();
+#pragma unroll
+                        for (int hu = 0; hu < 2; ++hu) {
+                            float v[16];
+                            load_acc16(tacc + acc0 + 32 * j + 16 * hu, v);
+                            add_bias16(v, bj, 16 * hu);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] = silu_f(v[i]);
+                            slabH_write16(sl, lane, hu, v);
+                        }
+                        slab_store(EMAP_A, sl, col0 + 32 * j, row0);
+                    }
+                } else if (mod) {
+                    // u = LN(h) * (1 + scale) + shift: operand of the next GEMM, leaves as bf16 slabs
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t sl = my_buf + (uint32_t)((u >> 1) & 1) * SLAB_H;
+                        if (u + 3 < 4) load_unit_h(P.h, chunk0, u + 3, lane, hin[(u + 3) & 3]);
+                        if ((u & 1) == 0) slab_ready();
+                        float sh[16], sc[16], hv[16];
+                        load_acc16(tacc + acc0 + 16 * u, sh);
+                        load_acc16(tacc + acc0 + 128 + 16 * u, sc);
+                        add_bias16(sh, (u >> 1) == 0 ? bq[0] : bq[1], 16 * (u & 1));
+                        add_bias16(sc, (u >> 1) == 0 ? bq[2] : bq[3], 16 * (u & 1));
+                        unit_h_values(hin[u & 3], hv);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) hv[i] = fmaf((hv[i] - mean) * rstd, 1.0f + sc[i], sh[i]);
+                        slabH_write16(sl, lane, u & 1, hv);
+                        if (u & 1) slab_store(EMAP_U, sl, col0 + 32 * (u >> 1), row0);
                     }
                 } else {
+                    // OP_G2: h += g * (acc + b2), read and written in place; LayerNorm partials of the 128 columns
                     Stats st;
-                    st.init(0.f);
-#pragma unroll 1
-                    for (int j = 0; j < io.nch && !fail; ++j) {
-                        const int b = j & 1;
-                        const uint32_t bufF = my_buf + (uint32_t)b * EPI_BUF;
-                        const uint32_t bufH = bufF + SLAB_F;
-                        if (has_loads) {
-                            if (j + 1 < io.nch) {
-                                // the other buffer was the source of the previous chunk's store
-                                if (lane == 0) ptx::bulk_wait_read<0>();
-                                issue_load(j + 1);
-                            }
-                            bool okw = wait_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u, P);
-                            okw = __all_sync(0xffffffffu, okw);
-                            fail |= !okw;
-                            if (fail) break;      // aborted: the load stays pending and is waited for at exit
-                            ld_parity ^= 1u << b;
-                            ld_pending &= ~(1u << b);
-                        } else {
-                            // the store that last used this buffer must have finished reading it
-                            if (lane == 0) ptx::bulk_wait_read<EPI_NB - 1>();
-                            __syncwarp();
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (u + 3 < 8) {
+                            load_unit_h(P.h, chunk0, u + 3, lane, hin[(u + 3) & 3]);
+                            load_unit_g(gsrc, chunk0, u + 3, lane, gin[(u + 3) & 3]);
                         }
-                        const float b0 = j == 0 ? bq[0] : j == 1 ? bq[1] : j == 2 ? bq[2] : bq[3];
-                        const float b1 = j == 0 ? bq[2] : bq[3];        // modulation items: the scale's bias
-                        epi_chunk(P, it, tacc + io.acc0 + 32 * j, io.acc0 + 32 * j, io.col0 + 32 * j, j == 0, bufF, bufH,
-                                  lane, st, mean, rstd, b0, b1);
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            if (io.stF >= 0) ptx::tma_store_2d(P.maps + io.stF, bufF, io.col0 + 32 * j, row0);
-                            if (io.stH >= 0) ptx::tma_store_2d(P.maps + io.stH, bufH, io.col0 + 32 * j, row0);
-                            ptx::bulk_commit();
-                        }
+                        float v[16], gv[16], hv[16];
+                        load_acc16(tacc + acc0 + 16 * u, v);
+                        add_bias16(v, (u >> 1) == 0 ? bq[0] : (u >> 1) == 1 ? bq[1] : (u >> 1) == 2 ? bq[2] : bq[3], 16 * (u & 1));
+                        unit_g_values(gin[u & 3], gv);
+                        unit_h_values(hin[u & 3], hv);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) hv[i] = fmaf(gv[i], v[i], hv[i]);
+                        if (u == 0) st.init(hv[0]);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) st.add(hv[i]);
+                        store_unit_h(P.h, chunk0, u, lane, hv);
                     }
-                    if (!fail && (it.type == OP_IN || it.type == OP_G2))
-                        P.stats[(size_t)grow * (2 * P.NT) + it.nt * 2 + half] = st.finish(128);
+                    P.stats[(size_t)grow * (2 * P.NT) + it.nt * 2 + half] = st.finish(128);
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive_even_cta(tempty_bar(buf));
                 ++acc_iter;
-                if (lane == 0) ptx::bulk_wait<0>();   // this warp's stores are performed
+                if (lane == 0) ptx::bulk_wait<0>();   // this warp's TMA stores are performed
                 __syncwarp();
             }
             if (fail) break;
@@ -967,9 +977,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
                 TRACE_NEXT();
             }
         }
-        // own copies in flight: loads that were issued but never consumed, stores not yet done
-        for (int b = 0; b < EPI_NB; ++b)
-            if (ld_pending & (1u << b)) drain_mbar(epi_bar(ew, b), (ld_parity >> b) & 1u);
+        // own copies in flight: stores not yet done
         if (lane == 0) ptx::bulk_wait<0>();
         __syncwarp();
     }
@@ -1348,7 +1356,7 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
     TRY(dev_alloc(H, &H->status, 2, true));
     TRY(dev_alloc(H, &H->clock_probe, 2, true));
 #ifdef ARDIFF_HEAD_PROFILE
-    TRY(dev_alloc(H, &H->trace, (size_t)TRACE_ITEMS * 3 * 4, true));
+    TRY(dev_alloc(H, &H->trace, (size_t)TRACE_ITEMS * 12 + (size_t)TRACE_ITEMS * 16, true));
 #endif
 
     // ---- the program of one step: phases in list order ----
@@ -1411,12 +1419,9 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, B_ROWS);
         ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, B_ROWS);
         ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C / 2);
-        ok &= make_slab_map(&maps[EMAP_H], H->h, R, W, true);
         ok &= make_slab_map(&maps[EMAP_S], H->s, (uint64_t)kmax * R, W, false);
         ok &= make_slab_map(&maps[EMAP_U], H->u, R, W, false);
         ok &= make_slab_map(&maps[EMAP_A], H->a, R, W, false);
-        ok &= make_slab_map(&maps[EMAP_G0], H->g0, R, W, false);
-        ok &= make_slab_map(&maps[EMAP_G1], H->g1, R, W, false);
         if (!ok) {
             free_all(H);
             delete H;
@@ -1620,7 +1625,7 @@ const ardiff_head_desc* head_desc(const ardiff_head* H) { return H ? &H->d : nul
 extern "C" int ardiff_head_copy_trace(ardiff_head* H, long long* dst, size_t count) {
     if (!H || !dst || !H->trace) return ARDIFF_ERR_NULL;
     if (cudaDeviceSynchronize() != cudaSuccess) return ARDIFF_ERR_CUDA;
-    if (count > (size_t)TRACE_ITEMS * 3 * 4) count = (size_t)TRACE_ITEMS * 3 * 4;
+    if (count > (size_t)TRACE_ITEMS * 28) count = (size_t)TRACE_ITEMS * 28;
     return cudaMemcpy(dst, H->trace, count * sizeof(long long), cudaMemcpyDeviceToHost) == cudaSuccess ? ARDIFF_OK
                                                                                                    : ARDIFF_ERR_CUDA;
 }

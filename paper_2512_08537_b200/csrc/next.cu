@@ -125,11 +125,16 @@ extern "C" int ardiff_entropy_gate_blocks(const void* feat, int64_t n, int32_t r
         ardiff::set_launch_count(1);
         return ardiff::write_zero_count(count, st);
     }
-    if (!feat || !row_entropy || !mask || !idx) return ARDIFF_ERR_NULL;
+    if (!feat || !mask || !idx) return ARDIFF_ERR_NULL;
     int32_t* counts = nullptr;
     int max_blocks = 0, sms = 0;
     int rc = ardiff::gate_scratch_get(st, &counts, &max_blocks, &sms);
     if (rc != ARDIFF_OK) return rc;
+    // one pass over the features when the shape allows it; else row entropies through global memory
+    rc = ardiff::gate_blocks_fused_launch(feat, n, rows_per_token, d, gamma, tau, row_entropy, token_entropy, mask,
+                                          idx, count, block_len, counts, max_blocks, sms, st);
+    if (rc != ARDIFF_ERR_UNSUPPORTED) return rc;
+    if (!row_entropy) return ARDIFF_ERR_NULL;      // this path needs it as scratch
     rc = ardiff::entropy_rows_launch(feat, n * rows_per_token, d, row_entropy, sms, st);
     if (rc != ARDIFF_OK) return rc;
     // CTAs own whole draft blocks, so a block never straddles two compaction ranges

@@ -158,3 +158,51 @@ def test_early_stop_feeds_accept_prefix_on_the_device():
     want = oracle.accept_prefix(r, ratio, 8, len_o)
     assert np.array_equal(got.cpu().numpy()[~band], want[~band])
     assert np.all(got.cpu().numpy() <= blen.cpu().numpy())
+
+
+def test_block_prefix_gate_without_row_entropy_output_and_on_the_two_pass_shape():
+    """The one-pass kernel keeps row entropies in shared memory (the caller need not take them); a draft
+    block whose rows exceed a CTA's shared memory goes through the row-entropy array instead and needs it."""
+    dev = require_cuda()
+    wl = synth.workload("cfg2", n=3000)
+    bits = synth.features(wl)
+    feat = dev_bf16(bits)
+    H = oracle.entropy(bits)
+    tau = float(np.quantile(H, 0.1))
+    a = ardiff.ardiff_entropy_gate_blocks(feat, 1, 8, tau, want_token_entropy=True)
+    b = ardiff.ardiff_entropy_gate_blocks(feat, 1, 8, tau, want_token_entropy=True, want_row_entropy=False)
+    torch.cuda.synchronize()
+    assert b[4] is None and torch.equal(a[0], b[0]) and torch.equal(a[3], b[3]) and torch.equal(a[5], b[5])
+    assert int(a[2].item()) == int(b[2].item())
+    # 30000 single-row tokens per draft block: beyond the one-pass limit
+    wl2 = synth.workload("cfg1", n=70001, d=64)
+    bits2 = synth.features(wl2)
+    tau2 = float(np.quantile(oracle.entropy(bits2), 0.0005))
+    check_blocks(bits2, 1, 30000, tau2)
+    with pytest.raises(ardiff.ArdiffError):
+        ardiff.ardiff_entropy_gate_blocks(dev_bf16(bits2), 1, 30000, tau2, want_row_entropy=False)
+
+
+@pytest.mark.parametrize("name,n,d", [("cfg2", 16384, 768), ("cfg4", 5000, 5120), ("cfg1", 77, 12)])
+def test_gate_with_threshold_statistics_in_one_pass(name, n, d):
+    """ardiff_entropy_gate_stats: the gate's usual outputs plus mean / std / tau of its own entropies."""
+    require_cuda()
+    wl = synth.workload(name, n=n, d=d)
+    bits = synth.features(wl)
+    feat = dev_bf16(bits)
+    H = oracle.entropy(bits)
+    tau = float(np.quantile(H, 0.3))
+    mask, idx, count, ent, out3 = ardiff.ardiff_entropy_gate_stats(feat, tau, want_entropy=True)
+    mask_p, idx_p, count_p, ent_p = ardiff.ardiff_entropy_gate(feat, tau, want_entropy=True)
+    torch.cuda.synchronize()
+    c = int(count.item())
+    assert c == int(count_p.item()) and torch.equal(mask, mask_p) and torch.equal(idx[:c], idx_p[:c])
+    assert torch.equal(ent, ent_p)
+    got = out3.cpu().numpy()
+    m, s, t = oracle.tau_calibrate(H)
+    assert abs(got[0] - m) <= 1e-3 and abs(got[1] - s) <= 1e-3 and abs(got[2] - t) <= 4e-4
+    # against the two-pass fp64 kernel on the very same fp32 entropies: only the summation order differs
+    ref = ardiff.ardiff_tau_calibrate(ent).cpu().numpy()
+    assert np.all(np.abs(got - ref) <= 1e-11)
+    again = ardiff.ardiff_entropy_gate_stats(feat, tau)[4].cpu().numpy()
+    assert np.array_equal(got, again)                                  # fixed merge order

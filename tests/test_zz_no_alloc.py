@@ -60,6 +60,26 @@ def test_noalloc_gate_matches_regular_gate_on_two_calls_in_a_row():
     assert _both(feat1, tau1) == kept1
 
 
+def test_noalloc_gate_leaves_device_memory_as_it_found_it():
+    """What the entry point is for: after its first call on the device (symbol look-up, kernel load), a call
+    takes no device memory: the driver's count of free bytes is the same before and after."""
+    require_cuda()
+    wl = synth.workload("cfg2", n=5000)
+    feat = dev_bf16(synth.features(wl))
+    dev = feat.device
+    mask = torch.empty((wl.n,), dtype=torch.uint8, device=dev)
+    idx = torch.empty((wl.n,), dtype=torch.int32, device=dev)
+    count = torch.empty((1,), dtype=torch.int32, device=dev)
+    ardiff.ardiff_entropy_gate_noalloc(feat, 5.0, mask, idx, count)          # first call for this row width
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for n in (5000, 1234):
+        ardiff.ardiff_entropy_gate_noalloc(feat[:n], 5.0, mask, idx, count)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+
+
 def test_noalloc_gate_rejects_sizes_beyond_its_fixed_capacity_and_handles_empty_input():
     dev = require_cuda()
     lib = ardiff.lib()
