@@ -37,7 +37,7 @@ NOMINAL_TFLOPS = 2250.0        # dense bf16, data sheet
 NOMINAL_HBM_GBS = 8000.0       # data sheet
 # dram__bytes_read.sum + dram__bytes_write.sum of one head_kernel launch, from the ncu captures summarised
 # under profiles/ (head_kernel_<workload>.txt); a workload without a capture of the current kernel reports null
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {"cfg4": 50.7e9, "cfg2": 4.09e9}
 
 
 def peaks():
@@ -196,6 +196,21 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
         return {"sm_mhz": statistics.median(self.samples), "sm_min_mhz": min(self.samples),
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+class L2Flush:
+    """Between timed iterations: 512 MiB written (every line of L2 replaced), then 256 MiB of other data
+    read, so that what L2 holds afterwards is unrelated AND clean. (After the write alone L2 is full of
+    dirty lines, and the next kernel pays for their write-back on top of its own traffic.)"""
+
+    def __init__(self, torch, dev):
+        self.torch = torch
+        self.w = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+        self.r = torch.zeros(L2_FLUSH_BYTES // 2, dtype=torch.uint8, device=dev)
+
+    def fill_(self, v):
+        self.w.fill_(v)
+        self.torch.max(self.r)
 
 
 def upload_bf16(torch, bits, dev):
@@ -400,7 +415,7 @@ def run_gpu(args, wl):
     if args.no_coop:
         head.set_cooperative(False)
     tau = quantile_tau(b.entropies(ardiff, torch), wl.filter_q)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush = L2Flush(torch, dev)
     stream = torch.cuda.current_stream()
     log("inputs resident")
 
@@ -444,6 +459,19 @@ def run_gpu(args, wl):
     ms_per_step = total_ms / args.steps
     value = world * n / (ms_per_step * 1e-3)
     log(f"burst: {ms_per_step:.3f} ms/step")
+
+    # ---- the gate by itself (gate + compaction launches), flushed before each call ----
+    gate_alone = []
+    for i in range(23):
+        flush.fill_(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ardiff.ardiff_entropy_gate(b.feat, tau, b.mask, b.idx, b.count, stream=stream)
+        e1.record(stream)
+        e1.synchronize()
+        if i >= 3:
+            gate_alone.append(e0.elapsed_time(e1))
+    gate_alone_ms = statistics.median(gate_alone)
 
     # ---- sustained: steps back to back for >= 2 s (inputs are larger than L2; no flush, no host sync) ----
     sus_iters = max(10, int(2200.0 / ms_per_step))
@@ -550,7 +578,8 @@ def run_gpu(args, wl):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "tokens_per_gpu": n, "survivors": S, "d": wl.d, "C": wl.C,
                        "Dc": wl.Dc, "W": wl.W, "L": wl.L, "K": wl.K, "tau": tau,
-                       "l2": "512 MiB written between timed iterations", "parallelism": f"dp{world}"},
+                       "l2": "512 MiB written, then 256 MiB of other data read, between timed iterations",
+                       "parallelism": f"dp{world}"},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                          "frac": achieved / pk["bf16_tflops"], "frac_nominal": achieved / NOMINAL_TFLOPS,
                          "nominal_peak": NOMINAL_TFLOPS,
@@ -572,7 +601,14 @@ def run_gpu(args, wl):
                                                "kernel_ms is the last launch of the loop"}},
             "gate": {"bound": "hbm", "achieved": gate_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": gate_gbs / pk["hbm_gbs"], "frac_nominal": gate_gbs / NOMINAL_HBM_GBS,
-                     "nominal_peak": NOMINAL_HBM_GBS, "ms": g_ms, "note": "gate + compaction launches"},
+                     "nominal_peak": NOMINAL_HBM_GBS, "ms": g_ms,
+                     "note": "gate + compaction launches, timed inside the steps (right before the head kernel, at "
+                             "the clock the power cap leaves)",
+                     "isolated": {"ms": gate_alone_ms,
+                                  "achieved": wl.gate_bytes() / (gate_alone_ms * 1e-3) / 1e9,
+                                  "frac": wl.gate_bytes() / (gate_alone_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                                  "frac_nominal": wl.gate_bytes() / (gate_alone_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                                  "note": "the same two launches alone, L2 flushed before each, median of 20"}},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_total / e2e_steps, "steps": e2e_steps,
                     "mode": "ardiff_pipeline_submit/_wait, 3 slots: copies overlap the kernels of the "
