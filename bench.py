@@ -368,6 +368,14 @@ def run_next_stage(torch, ardiff, dev, pk, flush, stream):
     ratio = torch.rand(n, device=dev) + 0.5
     rec("ardiff_accept_prefix gamma=8", f"{n} tokens", timed(lambda: ardiff.ardiff_accept_prefix(r_, ratio, 8)),
         8 * n + n // 8 * 4)
+    # row widths off the register path: long rows (one pass, running maximum) and a width that is no multiple of 8
+    for dd, nn in ((16384, 8192), (8200, 16384), (777, 65536)):
+        wl3 = synth.workload("cfg4", n=nn, d=dd)
+        f3 = upload_bf16(torch, synth.features(wl3), dev)
+        m3 = torch.empty(nn, dtype=torch.uint8, device=dev)
+        i3 = torch.empty(nn, dtype=torch.int32, device=dev)
+        rec("ardiff_entropy_gate", f"{nn} tokens x {dd}",
+            timed(lambda: ardiff.ardiff_entropy_gate(f3, 5.0, m3, i3, count)), nn * (2 * dd + 5) + 4)
     # attention-map-shaped input: 16 rows (heads x query rows) of 1024 keys per token
     wl2 = synth.workload("cfg3", n=4096 * 16)
     feat2 = upload_bf16(torch, synth.features(wl2), dev)

@@ -56,8 +56,9 @@ int ardiff_version(void);
  *   count  dev  int32 [1]  out: number of kept tokens (stays on the device)
  *   entropy (the _ex form) dev float [n] out, or NULL: H_i as computed
  *
- * Rows are read once from HBM (d <= 8192 and d % 8 == 0: registers hold the row; other d
- * take a slower two-pass kernel). n == 0 is valid (writes *count = 0).
+ * Rows are read once from HBM when d % 8 == 0 (d <= 8192: registers hold the row; longer rows:
+ * a running maximum per lane with rescaled partial sums); other d take a slower two-pass kernel
+ * with scalar loads. n == 0 is valid (writes *count = 0).
  *
  * Scratch and concurrency. The two kernels of a call hand per-block counts to each other
  * through a small per-device scratch (512 KB) that the library allocates on the first call on

@@ -273,6 +273,87 @@ gate_blocks_kernel(const uint4* __restrict__ feat, int64_t n_tokens, int32_t r, 
     }
 }
 
+// Rows longer than the registers hold (d > 8192, d % 8 == 0): still one pass with 128-bit loads. Every lane
+// keeps a running maximum of its own share of the row and rescales its partial sums when the maximum grows
+// (S <- S 2^D, T <- (T + D S) 2^D with D = (m_old - m_new) log2 e <= 0); the lanes' partials are merged the
+// same way at the end.
+__global__ void __launch_bounds__(kGateThreads)
+gate_rows_long_kernel(const uint4* __restrict__ feat, int64_t n, int32_t nchunks, float tau,
+                      uint8_t* __restrict__ mask, float* __restrict__ entropy,
+                      int32_t* __restrict__ block_counts, double* __restrict__ cta_stats, int64_t tokens_per_block) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.launch_dependents;");
+    const int64_t t_begin = (int64_t)blockIdx.x * tokens_per_block;
+    const int64_t t_end = min(n, t_begin + tokens_per_block);
+    int kept = 0;
+    WarpStats st{0.0, 0.0, 0.0};
+    for (int64_t tok = t_begin + warp; tok < t_end; tok += kGateWarps) {
+        const uint4* row = feat + tok * (int64_t)nchunks;
+        float ml = -CUDART_INF_F, S = 0.f, T = 0.f;
+        for (int c0 = lane; c0 < nchunks; c0 += 32 * 4) {
+            uint4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                v[j] = c0 + 32 * j < nchunks ? ld_stream_v4(row + c0 + 32 * j)
+                                             : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            uint32_t mx = 0xff80ff80u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                mx = max_bf16x2_nan(mx, max_bf16x2_nan(max_bf16x2_nan(v[j].x, v[j].y), max_bf16x2_nan(v[j].z, v[j].w)));
+            const float a = bf16_lo(mx), b = bf16_hi(mx);
+            const float mc = (a != a || b != b) ? CUDART_NAN_F : fmaxf(a, b);
+            if (mc != mc) ml = CUDART_NAN_F;
+            else if (mc > ml) {
+                if (S > 0.f) {
+                    const float D = (ml - mc) * kLog2e;
+                    const float f = ex2_approx(D);
+                    T = (T + D * S) * f;
+                    S = S * f;
+                }
+                ml = mc;
+            }
+            const float mneg = -ml * kLog2e;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (c0 + 32 * j < nchunks) {
+                    acc_word(v[j].x, mneg, S, T);
+                    acc_word(v[j].y, mneg, S, T);
+                    acc_word(v[j].z, mneg, S, T);
+                    acc_word(v[j].w, mneg, S, T);
+                }
+            }
+        }
+        const float m = warp_max_nan(ml);
+        if (S > 0.f && ml < m) {               // bring this lane's partials to the row maximum
+            const float D = (ml - m) * kLog2e;
+            const float f = ex2_approx(D);
+            T = (T + D * S) * f;
+            S = S * f;
+        }
+        S = warp_sum(S);
+        T = warp_sum(T);
+        float H = logf(S) - kLn2 * (T / S);
+        if (H != H) H = row_entropy_careful(row, nchunks, lane, m);
+        const bool keep = (H >= tau);
+        if (lane == 0) {
+            if (mask) mask[tok] = keep ? 1 : 0;
+            if (entropy) entropy[tok] = H;
+        }
+        kept += keep ? 1 : 0;
+        st.n += 1.0; st.s += (double)H; st.q += (double)H * (double)H;
+    }
+    __shared__ int s_cnt[kGateWarps];
+    if (lane == 0) s_cnt[warp] = kept;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int tot = 0;
+        for (int w = 0; w < kGateWarps; ++w) tot += s_cnt[w];
+        if (block_counts) block_counts[blockIdx.x] = tot;
+    }
+    if (cta_stats) cta_merge_stats(st, warp, lane, cta_stats + 3 * (size_t)blockIdx.x);
+}
+
 // Any d (no alignment assumption, any length): two passes over the row with scalar loads.
 __global__ void __launch_bounds__(kGateThreads)
 gate_rows_generic_kernel(const uint16_t* __restrict__ feat, int64_t n, int32_t d, float tau,
@@ -490,6 +571,9 @@ void launch_rows(int grid, cudaStream_t st, const void* feat, int64_t n, int32_t
             gate_rows_kernel<decltype(nch)::value><<<grid, kGateThreads, 0, st>>>(
                 reinterpret_cast<const uint4*>(feat), n, d / 8, tau, mask, entropy, counts, cta_stats, tpb);
         });
+    } else if (d % 8 == 0) {
+        gate_rows_long_kernel<<<grid, kGateThreads, 0, st>>>(reinterpret_cast<const uint4*>(feat), n, d / 8, tau, mask,
+                                                            entropy, counts, cta_stats, tpb);
     } else {
         gate_rows_generic_kernel<<<grid, kGateThreads, 0, st>>>(reinterpret_cast<const uint16_t*>(feat), n, d, tau,
                                                                mask, entropy, counts, cta_stats, tpb);
@@ -533,7 +617,7 @@ int grid_waves(int64_t rows, int32_t d, int64_t resident_blocks) {
 }
 
 int check_feat(const void* feat, int32_t d) {
-    const bool vec = (d % 8 == 0) && (d <= 8192);
+    const bool vec = (d % 8 == 0);
     if (vec && (reinterpret_cast<uintptr_t>(feat) & 15u)) return ARDIFF_ERR_ALIGN;
     if (!vec && (reinterpret_cast<uintptr_t>(feat) & 1u)) return ARDIFF_ERR_ALIGN;
     return ARDIFF_OK;

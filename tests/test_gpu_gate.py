@@ -75,7 +75,23 @@ def test_shapes_vector_path(n, d):
         check(bits, quantile_tau(H, q))
 
 
-@pytest.mark.parametrize("d", [1, 2, 7, 12, 777, 1001, 8200, 16384])
+@pytest.mark.parametrize("d", [8200, 12288, 16384, 65536])
+def test_shapes_long_rows_single_pass(d):
+    """Rows longer than the registers hold (d > 8192, d % 8 == 0): one pass with a running maximum per lane."""
+    wl = synth.workload("cfg4", n=41, d=d, seed=3000 + d)
+    bits = synth.features(wl)
+    H = oracle.entropy(bits)
+    for q in (0.0, 0.4):
+        check(bits, quantile_tau(H, q))
+    x = np.zeros((3, d), np.float32)
+    x[0, d - 5] = 90.0                    # the maximum arrives at the very end: every partial sum is rescaled
+    x[1, :d // 2] = -np.inf               # -inf channels contribute nothing
+    x[2, 4000] = np.nan                   # dropped
+    Hs, mask_g, _ = check(synth.f32_to_bf16(x), 0.5)
+    assert list(mask_g) == [0, 1, 0] and abs(Hs[1] - np.log(d - d // 2)) < 1e-9
+
+
+@pytest.mark.parametrize("d", [1, 2, 7, 12, 777, 1001, 8201, 16383])
 def test_shapes_generic_path(d):
     wl = synth.workload("cfg2", n=67, d=d, seed=2000 + d)
     bits = synth.features(wl)
