@@ -73,16 +73,14 @@ constexpr uint64_t kDrainLimitNs = 20000000ull;    // waits for own copies in fl
 #ifdef ARDIFF_HEAD_PROFILE
 constexpr int TRACE_ITEMS = 4096;
 #define TRACE(role, slot) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + (slot)] = clock64(); } while (0)
-#define TRACE_TYPE(role) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + 3] = it.type * 1000 + it.nt + ((role) == 0 ? 100 * trace_flag : 0); } while (0)
-#define TRACE_DECL int trace_n = 0; int trace_flag = 0;
-#define TRACE_FLAG(x) trace_flag = (x)
+#define TRACE_TYPE(role) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS) P.trace[((size_t)trace_n * 3 + (role)) * 4 + 3] = it.type * 1000 + it.nt; } while (0)
+#define TRACE_DECL int trace_n = 0;
 #define TRACE_NEXT() ++trace_n
 // per pipeline stage of the first 16 K slices of an item: role 0 = load issued, role 1 = MMA saw the stage full
 // (bit 0 of the stamp: it had to wait for it)
 #define TRACE_STAGE(role, kb) do { if (blockIdx.x == 0 && lane == 0 && P.trace && trace_n < TRACE_ITEMS / 2 && (kb) < 16) P.trace[(size_t)TRACE_ITEMS * 12 + ((size_t)trace_n * 16 + (kb)) * 2 + (role)] = clock64(); } while (0)
 #else
 #define TRACE_STAGE(role, kb)
-#define TRACE_FLAG(x)
 #define TRACE(role, slot)
 #define TRACE_TYPE(role)
 #define TRACE_DECL
