@@ -629,11 +629,21 @@ def run_gpu(args, wl):
             "gpu_launches": launches,
             "clocks": clocks,
         }
+        # the extra legs must never cost the main line: a failure is recorded in its place
         if world == 1 and not args.no_sweep:
-            line["sweep"] = run_sweep(torch, ardiff, dev, pk, flush, stream, wl, b, head, log)
-            line["next_stage"] = run_next_stage(torch, ardiff, dev, pk, flush, stream)
+            try:
+                line["sweep"] = run_sweep(torch, ardiff, dev, pk, flush, stream, wl, b, head, log)
+            except Exception as e:  # noqa: BLE001
+                line["sweep"] = {"error": f"{type(e).__name__}: {e}"}
+            try:
+                line["next_stage"] = run_next_stage(torch, ardiff, dev, pk, flush, stream)
+            except Exception as e:  # noqa: BLE001
+                line["next_stage"] = {"error": f"{type(e).__name__}: {e}"}
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(wl, weights, args.cpu_tokens, args.cpu_tokens_one_core)
+            try:
+                line["cpu_baseline"] = cpu_baseline(wl, weights, args.cpu_tokens, args.cpu_tokens_one_core)
+            except Exception as e:  # noqa: BLE001
+                line["cpu_baseline"] = {"error": f"{type(e).__name__}: {e}", "kind": "oracle"}
         print(json.dumps(line), flush=True)
     head.close()
     if dist is not None:
