@@ -642,7 +642,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) head_kernel(const __grid_const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { aborted = true; break; }
             TRACE(0, 0);
-            if (lane == 0) ptx::mbar_arrive(dep_bar(seq));      // the epilogue may now load this item's slabs
+            if (lane == 0) ptx::mbar_arrive(dep_bar(seq));      // the epilogue may now load this item's inputs
             ++seq;
             // operands that other CTAs wrote with plain stores (z, xb) cross from the generic to the async proxy;
             // everything else was written by TMA stores and is read by TMA loads
@@ -1100,19 +1100,17 @@ bool make_map(CUtensorMap* m, void* base, uint64_t rows, uint64_t cols, uint32_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// epilogue slab maps: box = [32 rows][32 columns]; fp32 rows are 128 B (128-byte swizzle), bf16 rows
-// 64 B (64-byte swizzle)
-bool make_slab_map(CUtensorMap* m, void* base, uint64_t rows, uint64_t cols, bool fp32) {
+// epilogue output slabs: bf16, box = [32 rows][32 columns], 64-byte rows, 64-byte swizzle
+bool make_slab_map(CUtensorMap* m, void* base, uint64_t rows, uint64_t cols) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
-    const uint64_t esz = fp32 ? 4 : 2;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * esz};
+    cuuint64_t strides[1] = {cols * 2};
     cuuint32_t box[2] = {32, 32};
     cuuint32_t estr[2] = {1, 1};
-    return fn(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides,
-              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, fp32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline float bf16_bits_to_float(uint16_t b) {
@@ -1417,9 +1415,9 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         ok &= make_map(&maps[MAP_WIN], H->Win, W, XB_COLS, B_ROWS);
         ok &= make_map(&maps[MAP_WCAT], H->Wcat, cat_rows, W, B_ROWS);
         ok &= make_map(&maps[MAP_WOUT], H->Wcat, cat_rows, W, (uint32_t)C / 2);
-        ok &= make_slab_map(&maps[EMAP_S], H->s, (uint64_t)kmax * R, W, false);
-        ok &= make_slab_map(&maps[EMAP_U], H->u, R, W, false);
-        ok &= make_slab_map(&maps[EMAP_A], H->a, R, W, false);
+        ok &= make_slab_map(&maps[EMAP_S], H->s, (uint64_t)kmax * R, W);
+        ok &= make_slab_map(&maps[EMAP_U], H->u, R, W);
+        ok &= make_slab_map(&maps[EMAP_A], H->a, R, W);
         if (!ok) {
             free_all(H);
             delete H;

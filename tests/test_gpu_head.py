@@ -338,10 +338,14 @@ def test_linear_sampler_steps(sampler):
 @pytest.mark.parametrize("shape", [dict(W=4096, L=1, K=1, C=32, Dc=64, n=130),
                                    dict(W=2048, L=2, K=2, C=64, Dc=128, n=300),
                                    dict(W=256, L=5, K=3, C=48, Dc=1024, n=257),
-                                   dict(W=512, L=1, K=64, C=16, Dc=64, n=40)])
+                                   dict(W=512, L=1, K=64, C=16, Dc=64, n=40),
+                                   dict(W=256, L=64, K=1, C=16, Dc=64, n=130),
+                                   dict(W=512, L=2, K=2, C=16, Dc=128, F=1024, n=200),
+                                   dict(W=256, L=2, K=3, C=32, Dc=64, F=2, n=129)])
 def test_extreme_shapes(shape):
     """Widest head (16 column tiles, 32 LayerNorm partials per row), the largest token dim, an odd number
-    of blocks (gate buffers alternate by block parity), the largest step count."""
+    of blocks (gate buffers alternate by block parity), the largest step count, the deepest head (64 blocks),
+    the largest and the smallest time-embedding size."""
     n = shape.pop("n")
     wl = synth.workload("cfg1", n=n, **shape)
     w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
@@ -378,4 +382,25 @@ def test_bounded_wait_runs_out_reports_timeout_and_the_head_recovers():
     with pytest.raises(ardiff.ArdiffError):
         head.inject_stall(0, 5)                           # limit below 100 us
     fresh.close()
+    head.close()
+
+
+def test_more_survivors_than_the_head_was_created_for():
+    """*count above max_tokens: the head runs the first max_tokens survivors, leaves every other row
+    untouched and flags the call with ARDIFF_ERR_SHAPE in its status word; the next call is clean."""
+    dev = require_cuda()
+    wl = synth.workload("cfg1", n=400)
+    w, cond_bits, noise, t = synth.head_weights(wl), synth.cond(wl), synth.noise(wl), synth.t_sched(wl.K)
+    head = make_head(wl, w, max_tokens=256)
+    idx_np = np.random.default_rng(2).permutation(wl.n)[:300].astype(np.int32)
+    want = oracle.head_sample(w, cond_bits, noise, t, idx_np[:256])
+    idx = torch.from_numpy(idx_np).to(dev)
+    count = torch.tensor([300], dtype=torch.int32, device=dev)
+    out = torch.full(noise.shape, SENTINEL, dtype=torch.float32, device=dev)
+    head.ardiff_head_sample(dev_bf16(cond_bits), dev_f32(noise), t, idx, count, out)
+    assert head.status() == ardiff.ARDIFF_ERR_SHAPE
+    got = out.cpu().numpy()
+    assert_parity(got, want, idx_np[:256])
+    assert np.all(got[np.setdiff1d(np.arange(wl.n), idx_np[:256])] == SENTINEL)
+    assert np.array_equal(run_head(head, cond_bits, noise, t, idx_np[:200])[idx_np[:200]], got[idx_np[:200]])
     head.close()
