@@ -206,8 +206,14 @@ typedef struct {
 
 /*
  * Packs the weights into the kernels' tile layout on the current device and allocates
- * the head's scratch (a fixed-size activation workspace sized to stay L2-resident plus
+ * the head's scratch (a fixed-size activation workspace for two groups of token tiles plus
  * max_tokens/128 progress counters). Synchronous; the only head call that allocates.
+ * Side effect on the CUDA context: while at least one head exists on a device, the context's
+ * cudaLimitPersistingL2CacheSize is at least the size of one token group's fp32 residual
+ * stream (about 49 MB, capped at the device's maximum); the kernel keeps that array in the
+ * persisting part of L2. The value found before the first head is put back when the last
+ * head of the device is destroyed, unless the caller changed the limit meanwhile. A device
+ * that refuses the limit runs the same kernel without that residency.
  * Errors: ERR_NULL, ERR_SHAPE / ERR_UNSUPPORTED for dims outside the ranges above,
  * ERR_NOMEM, ERR_CUDA (also when the device is not compute capability 10.x).
  */

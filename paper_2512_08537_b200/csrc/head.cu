@@ -33,6 +33,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "../../include/ardiff.h"
@@ -393,6 +394,10 @@ __device__ __forceinline__ void slabH_write16(uint32_t base, int r, int hu, cons
 // in chunk (row / 32, col / 32); inside the chunk the 16-byte piece p of the row's 32 columns of lane
 // row % 32 sits at 16-byte index p * 32 + lane. A 16-column unit u of a warp's span is pieces
 // 4 (u & 1) .. + 3 (fp32) or 2 (u & 1), + 1 (bf16) of chunk (first chunk + u / 2).
+// h is the one array that every residual block reads twice and writes once (three bytes of DRAM traffic per
+// byte held and block when it misses), and one group's h fits the part of L2 that a context may set aside for
+// persisting accesses: its loads and stores carry the evict_last policy, which keeps it there while the
+// bf16 operands stream past (ardiff_head_create sets that part aside).
 __device__ __forceinline__ size_t chunk_of(const HeadParams& P, int row0, int col0) {
     return (size_t)(row0 >> 5) * (size_t)(P.W >> 5) + (size_t)(col0 >> 5);
 }
@@ -400,13 +405,16 @@ struct UnitH { float4 p[4]; };      // 16 fp32 of one row
 struct UnitG { uint4 p[2]; };       // 16 bf16 of one row
 __device__ __forceinline__ void load_unit_h(const float* h, size_t chunk, int u, int lane, UnitH& d) {
     const float* src = h + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 4) * 128 + lane * 4;
+    const uint64_t pol = ptx::l2_evict_last_policy();
 #pragma unroll
-    for (int q = 0; q < 4; ++q) d.p[q] = ptx::ldcg_f4(src + q * 128);
+    for (int q = 0; q < 4; ++q) d.p[q] = ptx::ldcg_f4_hint(src + q * 128, pol);
 }
 __device__ __forceinline__ void store_unit_h(float* h, size_t chunk, int u, int lane, const float (&v)[16]) {
     float* dst = h + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 4) * 128 + lane * 4;
+    const uint64_t pol = ptx::l2_evict_last_policy();
 #pragma unroll
-    for (int q = 0; q < 4; ++q) ptx::st_f4(dst + q * 128, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
+    for (int q = 0; q < 4; ++q)
+        ptx::st_f4_hint(dst + q * 128, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]), pol);
 }
 __device__ __forceinline__ void load_unit_g(const bf16* g, size_t chunk, int u, int lane, UnitG& d) {
     const bf16* src = g + (chunk + (size_t)(u >> 1)) * 1024 + (size_t)((u & 1) * 2) * 256 + lane * 8;
@@ -1199,6 +1207,42 @@ int env_int(const char* name, int dflt) {
         }                           \
     } while (0)
 
+namespace {
+// The persisting part of L2 (a limit of the CUDA context, per device): raised while heads exist on the device
+// to what one token group's h needs, put back when the last of them is destroyed. A device or context that
+// refuses (no such part, MIG) leaves the kernel's evict_last hints without effect and nothing else changes.
+std::mutex g_l2_mu;
+struct L2SetAside { int users = 0; size_t before = 0, set = 0; };
+L2SetAside g_l2[64];
+
+void l2_set_aside_acquire(int dev, const cudaDeviceProp& prop, size_t want) {
+    if (dev < 0 || dev >= 64 || prop.persistingL2CacheMaxSize <= 0) return;
+    if (want > (size_t)prop.persistingL2CacheMaxSize) want = (size_t)prop.persistingL2CacheMaxSize;
+    std::lock_guard<std::mutex> lk(g_l2_mu);
+    L2SetAside& a = g_l2[dev];
+    size_t now = 0;
+    if (cudaDeviceGetLimit(&now, cudaLimitPersistingL2CacheSize) != cudaSuccess) { cudaGetLastError(); return; }
+    if (a.users == 0) { a.before = now; a.set = 0; }
+    ++a.users;
+    if (now < want) {
+        if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) != cudaSuccess) { cudaGetLastError(); return; }
+        cudaDeviceGetLimit(&a.set, cudaLimitPersistingL2CacheSize);
+    }
+}
+void l2_set_aside_release(int dev) {
+    if (dev < 0 || dev >= 64) return;
+    std::lock_guard<std::mutex> lk(g_l2_mu);
+    L2SetAside& a = g_l2[dev];
+    if (a.users == 0 || --a.users > 0 || a.set == 0) return;
+    size_t now = 0;
+    // only if nobody else has changed it since
+    if (cudaDeviceGetLimit(&now, cudaLimitPersistingL2CacheSize) == cudaSuccess && now == a.set)
+        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, a.before);
+    cudaGetLastError();
+    a.set = 0;
+}
+}  // namespace
+
 extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_head_host_weights* w,
                                   ardiff_head** head_out) {
     if (!desc || !w || !head_out) return ARDIFF_ERR_NULL;
@@ -1431,6 +1475,8 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         delete H;
         return ARDIFF_ERR_CUDA;
     }
+    // one token group's residual stream (half of the scratch rows, fp32)
+    l2_set_aside_acquire(dev, prop, (size_t)(H->slots / 2) * BM * (size_t)W * sizeof(float));
     *head_out = H;
     return ARDIFF_OK;
 }
@@ -1439,6 +1485,7 @@ extern "C" int ardiff_head_destroy(ardiff_head* H) {
     if (!H) return ARDIFF_OK;
     cudaSetDevice(H->device);
     cudaDeviceSynchronize();
+    l2_set_aside_release(H->device);
     if (H->ev0) cudaEventDestroy(H->ev0);
     if (H->ev1) cudaEventDestroy(H->ev1);
     free_all(H);

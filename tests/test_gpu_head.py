@@ -404,3 +404,32 @@ def test_more_survivors_than_the_head_was_created_for():
     assert np.all(got[np.setdiff1d(np.arange(wl.n), idx_np[:256])] == SENTINEL)
     assert np.array_equal(run_head(head, cond_bits, noise, t, idx_np[:200])[idx_np[:200]], got[idx_np[:200]])
     head.close()
+
+
+def test_persisting_l2_is_set_aside_while_a_head_exists_and_put_back_after():
+    # include/ardiff.h, ardiff_head_create: the context's persisting-L2 limit covers one token group's fp32
+    # residual stream while heads exist on the device, and returns to what it was with the last of them
+    rt = pytest.importorskip("cuda.bindings.runtime")
+    require_cuda()
+
+    def limit():
+        err, v = rt.cudaDeviceGetLimit(rt.cudaLimit.cudaLimitPersistingL2CacheSize)
+        assert int(err) == 0
+        return int(v)
+
+    err, max_size = rt.cudaDeviceGetAttribute(rt.cudaDeviceAttr.cudaDevAttrMaxPersistingL2CacheSize, 0)
+    assert int(err) == 0
+    if max_size <= 0:
+        pytest.skip("device has no persisting L2")
+    wl = synth.workload("cfg1")
+    weights = synth.head_weights(wl)
+    before = limit()
+    h1 = make_head(wl, weights)
+    during = limit()
+    group_h_bytes = 2 * 128 * wl.W * 4          # cfg1: one pair of token tiles per group
+    assert during >= min(group_h_bytes, max_size) and during >= before
+    h2 = make_head(wl, weights)
+    h1.close()
+    assert limit() == during
+    h2.close()
+    assert limit() == before
