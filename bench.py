@@ -37,7 +37,7 @@ NOMINAL_TFLOPS = 2250.0        # dense bf16, data sheet
 NOMINAL_HBM_GBS = 8000.0       # data sheet
 # dram__bytes_read.sum + dram__bytes_write.sum of one head_kernel launch, from the ncu captures summarised
 # under profiles/ (head_kernel_<workload>.txt); a workload without a capture of the current kernel reports null
-TRAFFIC_BYTES = {"cfg4": 50.7e9, "cfg2": 4.09e9}
+TRAFFIC_BYTES = {"cfg4": 37.4e9, "cfg2": 2.76e9}
 
 
 def peaks():
