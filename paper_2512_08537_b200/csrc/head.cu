@@ -23,9 +23,10 @@
 // (poll, vote, descriptors, two copies or four MMAs, commit) that takes most of the 512 cycles a slice lasts,
 // and they share their schedulers with two epilogue warps each (the TMEM lane quarter a warp may read is its
 // id modulo 4, so every scheduler hosts the epilogue of one quarter). Every slot an epilogue warp takes there
-// lengthens the chain; the ring drains and the tensor pipe waits. Measured on copies of this kernel that skip
-// work: without any epilogue work a slice is consumed every 545 cycles and the launch takes 21 % fewer cycles;
-// with a sixteenth of the operand bytes it takes 4 % fewer. So the kernel keeps the two chains and the
+// lengthens the chain, and the epilogue's own loads and stores compete with the copies; the ring drains and
+// the tensor pipe waits. Measured on copies of this kernel that skip work: without any epilogue work a slice
+// is consumed every 545 cycles and the launch takes 21 % fewer cycles (8 points of that are the epilogue's
+// memory operations); with a sixteenth of the operand bytes it takes 4 % fewer. So the kernel keeps the two chains and the
 // epilogue short: biases travel in registers (one column per lane, handed round by shuffle), c never leaves
 // the accumulator, epilogue inputs are plain loads issued three units ahead, h and the gate values stay off
 // shared memory, and proxy fences sit only where a proxy is really crossed.
