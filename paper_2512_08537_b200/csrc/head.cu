@@ -1324,6 +1324,11 @@ extern "C" int ardiff_head_create(const ardiff_head_desc* desc, const ardiff_hea
         if (tg_env > 0) tgu = tg_env;
     }
 #endif
+    // A unit gets r = ceil(tgu * NT / units) in-projection items in a row, each a single K slice: the producer can
+    // then be r + 1 items ahead of the MMA issuer, which with its two accumulators is up to 2 ahead of the
+    // epilogue; the dependency barriers are a ring of DEP_BARS phases, so r + 3 must stay below DEP_BARS
+    // (r = 3 with the group size chosen above).
+    while (tgu > 1 && ((int64_t)tgu * NT + units - 1) / units > DEP_BARS - 4) --tgu;
     if (tgu < 1) tgu = 1;
     if ((int64_t)tgu * 2 > H->max_tiles + 1) tgu = (int)((H->max_tiles + 1) / 2);
     H->TGu = tgu;
